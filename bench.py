@@ -1,0 +1,299 @@
+#!/usr/bin/env python
+"""Benchmark of the OD-SGD parameter-update pass.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--workers M]
+    python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+A step is one OD-SGD iteration of the update pass on one synthetic parameter set: the fused
+global + local update (server step over M gradient buffers plus one worker's local weights)
+in a single kernel launch.  `value` is algorithmic bytes per second, (M + 5) * 4 * P bytes per
+step, with every buffer resident in HBM; `e2e` is the same figure when the M gradients start
+in pinned host memory and the worker's new weights are copied back, all inside the timed
+region, through the host-buffer entry point of the C ABI.  One JSON line goes to stdout.
+
+With --gpus N > 1 (under torchrun) every rank updates its own full parameter set on its own
+GPU: the ranks share no data, so nothing but a barrier and the final max/sum of two scalars
+crosses between them.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "OD-SGD update throughput: HBM GB/s & % of B200 peak; params/sec at N workers"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--workload", default="vgg16", help="lenet5 | resnet56 | alexnet | resnet50 | vgg16")
+    ap.add_argument("--workers", type=int, default=0, help="override the workload's worker count")
+    ap.add_argument("--deterministic", action="store_true", help="time the one-rounding-per-operator flavour")
+    ap.add_argument("--block", type=int, default=0)
+    ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra-kernels", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="elements in the oracle's sample")
+    return ap.parse_args()
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+def oracle_sample(wl, n_workers, sample_elems):
+    """Inputs for the oracle: the workload's hyper-parameters and value distributions on an
+    arena cut down to `sample_elems` elements."""
+    import numpy as np
+
+    from paper_2005_06728_b200 import workloads as W
+
+    s = min(sample_elems, wl.arena_len)
+    cut = W.ragged_workload([s], n_workers, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum,
+                            wd=wl.wd, seed=wl.seed, name=wl.name + "-sample")
+    cut.grad_sigma = wl.grad_sigma
+    rng_w = W.make_weights(wl if wl.arena_len <= (1 << 24) else cut)
+    w = rng_w[:s].numpy().copy()
+    v = np.zeros(s, np.float32)
+    grads = [W.make_grad(cut, m, 0).numpy() for m in range(n_workers)]
+    return cut, w, v, grads
+
+
+def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
+    """Times the oracle as it stands (single thread) on the sample; returns (GB/s, info)."""
+    import numpy as np
+
+    import oracle
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes, host_info
+
+    cut, w, v, grads = oracle_sample(wl, n_workers, sample_elems)
+    s = w.size
+    wp = np.empty_like(w)
+    x = np.empty_like(w)
+    times = []
+    t_start = time.perf_counter()
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle.global_update(grads, w, v, lr=wl.lr, momentum=wl.momentum, wd=wl.wd, w_prev=wp)
+        oracle.local_update(wp, grads[0], local_lr=wl.local_lr, out=x)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+        if it >= warmup + 2 and time.perf_counter() - t_start > budget_s:
+            break
+    sec = statistics.mean(times)
+    nbytes = algorithmic_bytes("fused", s, n_workers)
+    info = {"value": nbytes / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"first {s} of {wl.arena_len} elements of {wl.name}, all {n_workers} workers, "
+                      f"{len(times)} calls of global+local update, single thread",
+            "ms_per_call": sec * 1e3, "params_per_s": s / sec, "host": host_info()}
+    return info, len(times), sec
+
+
+def run_reference(args):
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import rank_info
+
+    if rank_info()["rank"] != 0:
+        return 0
+    wl = W.workload(args.workload)
+    n_workers = args.workers or wl.n_workers
+    info, done, sec = time_oracle(wl, n_workers, args.cpu_sample, args.steps, args.warmup, budget_s=150.0)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": info["value"], "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": done, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name} M={n_workers} (CPU oracle on a bounded sample)", "n_params": wl.n_params,
+                   "n_workers": n_workers, "sample_elems": min(args.cpu_sample, wl.arena_len)},
+        "cpu_baseline": {k: info[k] for k in ("value", "unit", "cores", "kind", "sample")},
+        "e2e": {"value": info["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "params_per_s": info["params_per_s"], "host": info["host"],
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    import torch
+
+    from paper_2005_06728_b200 import binding
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import (ClockSampler, aggregate, algorithmic_bytes, barrier,
+                                                 init_process_group, rank_info)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the update pass has no CPU path")
+    binding.load_library()  # fail now if the CUDA library is missing
+    ri = rank_info()
+    world = ri["world_size"]
+    if world > 1:
+        init_process_group("nccl")
+    dev = torch.device("cuda", ri["local_rank"] if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    rank0 = ri["rank"] == 0
+
+    wl = W.workload(args.workload)
+    M = args.workers or wl.n_workers
+    n, P = wl.arena_len, wl.n_params
+    free, total = torch.cuda.mem_get_info()
+    need = (M + 5) * n * 4
+    if need > 0.9 * free:
+        raise SystemExit(f"{wl.name} with {M} workers needs {need / 2**30:.1f} GiB; {free / 2**30:.1f} GiB free")
+
+    w_a = W.make_weights(wl, dev)
+    w_b = torch.zeros_like(w_a)
+    v = W.make_momentum(wl, dev)
+    local = [torch.zeros_like(w_a)] + [None] * (M - 1)
+    sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
+    grads = [W.make_grad(wl, m, 0, dev, _sigma=sg, _pads=pads) for m in range(M)]
+    flags = binding.FLAG_DETERMINISTIC if args.deterministic else 0
+    ctx = binding.Odsgd(w_a, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                        w_b=w_b, local=local, tensor_offsets=wl.offsets, flags=flags)
+    if args.block or args.ctas_per_sm:
+        ctx.set_launch_config(args.block, args.ctas_per_sm)
+    stream = torch.cuda.current_stream()
+
+    step_bytes = algorithmic_bytes("fused", P, M)
+    l2_note = ("inputs per step exceed the 126 MB L2 many times over: no flush" if step_bytes > 8 * 126e6
+               else "working set fits in L2: effective GB/s, not an HBM figure")
+
+    for _ in range(max(3, args.warmup)):
+        ctx.fused_update(grads, 0, stream)
+    torch.cuda.synchronize()
+    barrier(dev)
+    torch.cuda.synchronize()
+    launches_before = ctx.launch_count
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    with ClockSampler(dev.index or 0) as clocks:
+        ev[0].record(stream)
+        for k in range(args.steps):
+            ctx.fused_update(grads, 0, stream)
+            ev[k + 1].record(stream)
+        torch.cuda.synchronize()
+    barrier(dev)
+    torch.cuda.synchronize()
+    gpu_launches = ctx.launch_count - launches_before
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    agg = aggregate(total_ms, float(step_bytes) * args.steps, dev if world > 1 else None)
+    ms_per_step = agg["ms"] / args.steps
+    value = agg["units"] / (agg["ms"] * 1e-3) / 1e9
+    kernel_ms = total_ms / args.steps  # one launch per step, back to back on one stream
+    achieved = step_bytes / (kernel_ms * 1e-3) / 1e9
+    peak, peak_src = hbm_peak()
+
+    # ---- the other rules on the same arena (context only; not part of `value`)
+    extra = {}
+    if not args.no_extra_kernels and rank0:
+        def timed(fn, reps):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        reps = max(5, min(50, args.steps))
+        for name, fn in (("global", lambda: ctx.global_update(grads, stream)),
+                         ("local", lambda: ctx.local_update(0, stream)),
+                         ("ssgd", lambda: ctx.ssgd_step(grads, stream)),
+                         ("asgd", lambda: ctx.asgd_step(0, grads[0], stream))):
+            if name == "local":
+                ctx.global_update(grads, stream)
+            ms = timed(fn, reps)
+            b = algorithmic_bytes(name, P, M)
+            extra[name] = {"ms": ms, "GBps": b / ms / 1e6, "frac": b / ms / 1e6 / peak}
+
+    # ---- end to end: gradients start in pinned host memory, local weights come back
+    e2e = None
+    if not args.no_e2e:
+        pool = [W.make_grad(wl, m, 1, dev, _sigma=sg, _pads=pads).cpu().pin_memory() for m in range(min(M, 4))]
+        host_grads = [pool[m % len(pool)] for m in range(M)]
+        host_out = torch.empty(n, dtype=torch.float32).pin_memory()
+        e2e_steps = max(2, min(args.steps, 6))
+        ctx.fused_update_host(host_grads, grads, 0, host_out, stream)
+        torch.cuda.synchronize()
+        barrier(dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.perf_counter()
+        a.record(stream)
+        for _ in range(e2e_steps):
+            ctx.fused_update_host(host_grads, grads, 0, host_out, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        e2e_ms = max(a.elapsed_time(b), wall_ms)
+        agg2 = aggregate(e2e_ms, float(step_bytes) * e2e_steps, dev if world > 1 else None)
+        e2e = {"value": agg2["units"] / (agg2["ms"] * 1e-3) / 1e9, "unit": "GB/s",
+               "h2d_bytes_per_step": M * n * 4, "d2h_bytes_per_step": n * 4, "steps": e2e_steps,
+               "ms_per_step": agg2["ms"] / e2e_steps,
+               "note": f"{M} host-to-device copies per step from a pool of {len(pool)} distinct pinned buffers"}
+
+    if not rank0:
+        return 0
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        info, _, _ = time_oracle(wl, M, args.cpu_sample, steps=10, warmup=1)
+        cpu = {k: info[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        cpu["host"] = info["host"]
+
+    ck = clocks.summary()
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name}-shaped parameter set, M={M} workers, fused global+local update",
+                   "n_params": P, "n_tensors": wl.n_tensors, "n_workers": M,
+                   "bytes_per_step": step_bytes, "l2": l2_note,
+                   "flavour": "deterministic" if args.deterministic else "default (FMA contraction allowed)",
+                   "parallelism": "independent replicas" if world > 1 else "single GPU"},
+        "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),
+                   "power_w_max": ck.get("power_w_max"), "samples": ck.get("samples"), "source": ck.get("source")},
+        "e2e": e2e, "gpu_launches": gpu_launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": f"of {peak_src}", "kernel": "server_kernel (fused, one local)",
+                     "kernel_ms": kernel_ms, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
+        "cpu_baseline": cpu,
+        "params_per_s": P * args.steps * world / (agg["ms"] * 1e-3),
+        "grad_elems_per_s": M * P * args.steps * world / (agg["ms"] * 1e-3),
+        "step_ms": {"median": statistics.median(per_step), "min": min(per_step), "max": max(per_step)},
+        "other_kernels": extra,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

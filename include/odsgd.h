@@ -1,0 +1,235 @@
+/*
+ * odsgd.h - C ABI of the OD-SGD parameter-update library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the per-iteration parameter-update pass of One-step Delay SGD
+ * (OD-SGD) and of the two rules the paper compares it with (SSGD, ASGD) as fused
+ * one-pass CUDA kernels over a flat fp32 parameter arena:
+ *
+ *   - the GLOBAL update, the parameter-server role (paper: Algorithm 1, "Update w_t
+ *     with aggregated gradient" once all M workers have delivered):
+ *         gbar = (g_0 + g_1 + ... + g_{M-1}) * (1/M)     workers added in this order
+ *         d    = gbar + wd * w
+ *         v'   = momentum * v - lr * d
+ *         w'   = w + v'
+ *   - the LOCAL update, the worker role (paper: Algorithm 2, repeat-loop, "w_bak = w_t"
+ *     then "Update w_bak with g_m"; Section 3.3 "Local Updater"):
+ *         x_m  = w_bak - local_lr * g_m
+ *     where w_bak is the global weight vector from BEFORE this iteration's global
+ *     update (the worker has not pulled the new one yet); x_m are the weights worker
+ *     m trains on next.  Delay-compensated flavours: Eq. 4 and Eq. 5/6.
+ *   - the SSGD server step (Section 3.1: the server side is the same as OD-SGD's) and
+ *     the ASGD server step (Section 1: each arriving gradient is applied at once).
+ *
+ * Conventions
+ *   - Every function returns an int: ODSGD_OK (0) or a negative ODSGD_ERR_* code.
+ *     Nothing throws across this boundary.  odsgd_last_error() gives a text for the
+ *     most recent failure on a context.
+ *   - "device pointer" = address in the memory of the CUDA device that was current
+ *     when odsgd_create() ran; "host pointer" = ordinary process memory.
+ *   - The caller owns every device buffer for the whole life of the context; the
+ *     context only borrows them.  The library allocates no parameter-sized memory.
+ *   - All update calls are asynchronous: they enqueue work on `stream` (a
+ *     cudaStream_t passed as void*; NULL = the legacy default stream) and return.
+ *     The library never synchronises.  Buffers must stay valid until that work is done.
+ *   - Arena layout: all parameter tensors concatenated into one float array of
+ *     `n_params` elements; `tensor_offsets` (n_tensors + 1 ascending element offsets,
+ *     first 0, last n_params) marks where each tensor starts.  Gradient arenas, the
+ *     momentum arena and the local-weight arenas use the same layout.  Padding
+ *     elements between tensors are updated like any other element (zeros stay zeros).
+ *   - Alignment: the fast path needs every device pointer 16-byte aligned.  Without
+ *     ODSGD_FLAG_ALLOW_UNALIGNED a misaligned pointer is rejected with ODSGD_ERR_ALIGN;
+ *     with it, a scalar (4-byte) kernel is used for that call.
+ *   - Arithmetic is IEEE-754 binary32, round-to-nearest-even, subnormals kept.  By
+ *     default the compiler may fuse a multiply with the following add (one rounding
+ *     instead of two).  With ODSGD_FLAG_DETERMINISTIC every operator written above
+ *     rounds on its own, so results are reproducible bit for bit against a plain
+ *     scalar CPU evaluation in the same order.
+ */
+#ifndef ODSGD_H_
+#define ODSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ODSGD_VERSION_MAJOR 0
+#define ODSGD_VERSION_MINOR 1
+
+/* Largest number of workers (gradient buffers) one context can take. */
+#define ODSGD_MAX_WORKERS 64
+
+#define ODSGD_OK 0
+#define ODSGD_ERR_ARG (-1)         /* NULL where a pointer is needed, size or index out of range */
+#define ODSGD_ERR_ALIGN (-2)       /* a device pointer is not 16-byte aligned (4-byte for the scalar path) */
+#define ODSGD_ERR_OVERLAP (-3)     /* two buffers that must be distinct overlap */
+#define ODSGD_ERR_STATE (-4)       /* call not valid in the context's current state */
+#define ODSGD_ERR_CUDA (-5)        /* a CUDA runtime call or the launch failed; text in odsgd_last_error */
+#define ODSGD_ERR_UNSUPPORTED (-6) /* valid request this build does not implement */
+
+#define ODSGD_FLAG_DETERMINISTIC 0x1u   /* no fused multiply-add: one rounding per operator */
+#define ODSGD_FLAG_ALLOW_UNALIGNED 0x2u /* accept 4-byte aligned pointers (slower scalar kernel) */
+
+/* Local update rules (Section 3.3, "Local Updater"). */
+#define ODSGD_LOCAL_SGD 0  /* x = w_bak - local_lr * g */
+#define ODSGD_LOCAL_DC_C 1 /* Eq. 4 */
+#define ODSGD_LOCAL_DC_A 2 /* Eq. 5 with the running mean square of Eq. 6 */
+
+typedef struct odsgd_ctx odsgd_ctx;
+
+/*
+ * Description of one training job's parameter state.  Plain data, copied by
+ * odsgd_create(); the arrays it points to (local, tensor_offsets) are host arrays
+ * read during the call only.
+ *
+ * Weight storage, two layouts:
+ *   ping-pong  (w_b != NULL): each global update reads the current half and writes
+ *              the other one, then the halves swap roles.  The half just read still
+ *              holds the old weights, which are exactly the w_bak the workers need,
+ *              so keeping them costs no extra traffic.  w_delayed must be NULL.
+ *   in place   (w_b == NULL): the global update overwrites w_a.  If w_delayed != NULL
+ *              the old weights are also written there (one extra store stream) so
+ *              that odsgd_local_update() can run later; if it is NULL only the fused
+ *              call can produce local weights.
+ */
+typedef struct odsgd_desc {
+    float* w_a;                   /* device, n_params floats: global weights w_0 at create time */
+    float* w_b;                   /* device, n_params floats, or NULL */
+    float* w_delayed;             /* device, n_params floats, or NULL (in-place layout only) */
+    float* v;                     /* device, n_params floats: momentum state (caller zero-fills for a fresh run) */
+    float* const* local;          /* host array of n_workers device pointers (entries may be NULL), or NULL */
+    size_t n_params;              /* elements in each arena, > 0 */
+    const size_t* tensor_offsets; /* host, n_tensors + 1 ascending offsets, [0] = 0, [n_tensors] = n_params */
+    size_t n_tensors;             /* >= 1 */
+    int n_workers;                /* M, 1 .. ODSGD_MAX_WORKERS */
+    float lr;                     /* global learning rate */
+    float local_lr;               /* local learning rate */
+    float momentum;
+    float wd;                     /* weight decay (L2 coefficient) */
+    uint32_t flags;               /* ODSGD_FLAG_* */
+} odsgd_desc;
+
+/* Library version as major * 1000 + minor. */
+int odsgd_version(void);
+
+/* Text for an ODSGD_ERR_* code (static storage). */
+const char* odsgd_strerror(int code);
+
+/*
+ * Validates `desc` and builds a context on the current CUDA device.  No kernel is
+ * launched and nothing is written to the caller's buffers.
+ * Errors: ERR_ARG (NULL/zero/out-of-range field, offsets not ascending or not ending
+ * at n_params, w_delayed given together with w_b), ERR_ALIGN, ERR_OVERLAP (any two of
+ * w_a, w_b, w_delayed, v, local[m] overlap), ERR_CUDA (no usable device).
+ * On error *out is set to NULL; odsgd_last_error(NULL) describes the failure.
+ */
+int odsgd_create(odsgd_ctx** out, const odsgd_desc* desc);
+
+/* Frees the context (host memory and its small device tables).  Caller buffers are untouched. */
+int odsgd_destroy(odsgd_ctx* ctx);
+
+/*
+ * Global update (Algorithm 1).  `worker_grads` is a HOST array of n_workers DEVICE
+ * pointers, each an arena of n_params floats; they are read only and summed in index
+ * order.  Advances the step counter; in the ping-pong layout swaps the halves.  The
+ * gradient pointers are remembered as "this iteration's gradients" so that
+ * odsgd_local_update() can follow.
+ * Errors: ERR_ARG (NULL table or entry), ERR_ALIGN, ERR_OVERLAP (a gradient buffer
+ * overlaps a state buffer), ERR_CUDA.
+ */
+int odsgd_global_update(odsgd_ctx* ctx, const float* const* worker_grads, void* stream);
+
+/*
+ * Local update of worker `worker_id` (Algorithm 2, "Update w_bak with g_m"):
+ * local[worker_id] = w_bak (-) local_lr * g_worker_id, with w_bak the weights from
+ * before the latest odsgd_global_update() and g the gradient bound by that call
+ * (the gradient buffer must still hold the same data).
+ * Errors: ERR_STATE (no global update since create or since the last SSGD/ASGD step,
+ * or in-place layout without w_delayed), ERR_ARG (worker_id out of range, or no local
+ * buffer for that worker).
+ */
+int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream);
+
+/*
+ * Fused global + local update: the global update and the local update of one worker
+ * (worker_id >= 0) or of every worker that has a local buffer (worker_id == -1) in a
+ * single pass; the weights and each gradient are read once.  Results are bit-identical
+ * to odsgd_global_update() followed by odsgd_local_update().  Same state effects and
+ * errors as those two calls.
+ */
+int odsgd_fused_update(odsgd_ctx* ctx, const float* const* worker_grads, int worker_id, void* stream);
+
+/*
+ * Same as odsgd_fused_update() for gradients that arrive in HOST memory (as they do at
+ * a parameter server fed by a network).  `host_grads`: host array of n_workers host
+ * pointers (page-locked memory for real asynchrony), n_params floats each.
+ * `dev_staging`: host array of n_workers device pointers the gradients are copied
+ * into (caller-owned, n_params floats each).  If `host_local_out` is not NULL and
+ * worker_id >= 0, local[worker_id] is copied back to it after the update.  All copies
+ * and the kernel are enqueued on `stream` in order; nothing is synchronised.
+ */
+int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging,
+                            int worker_id, float* host_local_out, void* stream);
+
+/*
+ * SSGD server step (Section 3.1): the same arithmetic as the global update, applied
+ * in place to the current weights; no backup weights are kept and no local update may
+ * follow (workers pull the new weights instead).
+ */
+int odsgd_ssgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream);
+
+/*
+ * ASGD server step (Section 1): one worker's gradient `grad` (device pointer) is
+ * applied at once, without sum or 1/M: d = g + wd*w; v' = momentum*v - lr*d; w' = w + v'.
+ * In place on the current weights.  `worker_id` (0 .. n_workers-1) is recorded only;
+ * the order of application is the order of the calls.
+ */
+int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream);
+
+/* Hyper-parameters are kernel arguments, so schedules may change them before any call. */
+int odsgd_set_lr(odsgd_ctx* ctx, float lr);
+int odsgd_set_local_lr(odsgd_ctx* ctx, float local_lr);
+int odsgd_set_momentum(odsgd_ctx* ctx, float momentum);
+int odsgd_set_wd(odsgd_ctx* ctx, float wd);
+
+/*
+ * Chooses the local update rule (Section 3.3).  ODSGD_LOCAL_SGD ignores the other
+ * arguments.  ODSGD_LOCAL_DC_C uses `lambda` (Eq. 4).  ODSGD_LOCAL_DC_A uses `lambda`,
+ * the mean-square decay `m` and `eps` (Eq. 5, Eq. 6) and needs one mean-square arena
+ * per worker with a local buffer: `mean_square` is a host array of n_workers device
+ * pointers (n_params floats each, caller-owned and caller-initialised, normally zeros);
+ * pass NULL for the other rules.  In both delay-compensated rules the vector the
+ * gradient was computed on (the paper's w_t) is the worker's previous local weights,
+ * i.e. the content of local[worker] before the call, which is then overwritten.
+ */
+int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float eps,
+                         float* const* mean_square);
+
+/* Current and backup (one step old) weight arenas; either output pointer may be NULL.
+ * *delayed is NULL when the context keeps no backup or none is valid yet. */
+int odsgd_get_weights(odsgd_ctx* ctx, float** current, float** delayed);
+
+/* Number of global updates (OD-SGD or SSGD) plus ASGD steps applied so far. */
+int odsgd_get_step(odsgd_ctx* ctx, uint64_t* step);
+int odsgd_set_step(odsgd_ctx* ctx, uint64_t step);
+
+/*
+ * Launch shape of the update kernels.  block_threads: 64..1024, multiple of 32;
+ * ctas_per_sm: >= 1, grid = min(tiles, SMs * ctas_per_sm) persistent CTAs; 0 for
+ * either restores the built-in choice.
+ */
+int odsgd_set_launch_config(odsgd_ctx* ctx, int block_threads, int ctas_per_sm);
+
+/* How many kernels this context has launched since create. */
+int odsgd_get_launch_count(odsgd_ctx* ctx, uint64_t* launches);
+
+/* Text describing the last failure on `ctx` (or, for ctx == NULL, of the last failed
+ * odsgd_create on this thread).  Never NULL. */
+const char* odsgd_last_error(odsgd_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ODSGD_H_ */

@@ -1,0 +1,622 @@
+// Host side of the OD-SGD update library: context, validation, kernel selection
+// and launches behind the C ABI declared in odsgd.h.  No torch types, no
+// allocation of parameter-sized memory, no synchronisation.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "odsgd.h"
+#include "odsgd_kernels.cuh"
+
+using namespace odsgd;
+
+struct odsgd_ctx {
+    int device = 0;
+    int sm_count = 0;
+    float* w[2] = {nullptr, nullptr};
+    int cur = 0;  // index of the half that holds the current weights
+    bool pingpong = false;
+    float* w_delayed = nullptr;  // in-place layout: optional backup arena
+    float* v = nullptr;
+    float* local[ODSGD_MAX_WORKERS] = {};
+    float* mean_square[ODSGD_MAX_WORKERS] = {};
+    size_t n = 0;
+    std::vector<size_t> offsets;
+    int n_workers = 0;
+    float lr = 0, local_lr = 0, momentum = 0, wd = 0;
+    uint32_t flags = 0;
+    int local_rule = ODSGD_LOCAL_SGD;
+    float dc_lambda = 0, dc_m = 0, dc_eps = 0;
+    const float* bound[ODSGD_MAX_WORKERS] = {};  // gradients of the latest global update
+    bool grads_bound = false;
+    const float* delayed = nullptr;  // weights from before the latest global update, if kept
+    uint64_t step = 0;
+    uint64_t launches = 0;
+    int block_threads = 0;  // 0 = built-in
+    int ctas_per_sm = 0;    // 0 = built-in
+    std::string err;
+};
+
+namespace {
+
+thread_local std::string g_create_err;
+
+constexpr int kDefaultBlock = 256;
+
+int fail(odsgd_ctx* ctx, int code, const std::string& msg) {
+    if (ctx) ctx->err = msg; else g_create_err = msg;
+    return code;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+bool overlap(const void* a, const void* b, size_t bytes) {
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + bytes && y < x + bytes;
+}
+
+struct Named {
+    const void* p;
+    const char* name;
+    int idx;
+};
+
+std::string label(const Named& b) {
+    char buf[64];
+    if (b.idx >= 0) snprintf(buf, sizeof buf, "%s[%d]", b.name, b.idx); else snprintf(buf, sizeof buf, "%s", b.name);
+    return buf;
+}
+
+// State buffers of a context, for alias checks.
+std::vector<Named> state_buffers(const odsgd_ctx* c) {
+    std::vector<Named> s;
+    s.push_back({c->w[0], "w_a", -1});
+    if (c->w[1]) s.push_back({c->w[1], "w_b", -1});
+    if (c->w_delayed) s.push_back({c->w_delayed, "w_delayed", -1});
+    s.push_back({c->v, "v", -1});
+    for (int m = 0; m < c->n_workers; ++m) {
+        if (c->local[m]) s.push_back({c->local[m], "local", m});
+        if (c->mean_square[m]) s.push_back({c->mean_square[m], "mean_square", m});
+    }
+    return s;
+}
+
+int check_distinct(odsgd_ctx* err_ctx, const std::vector<Named>& s, size_t bytes) {
+    for (size_t i = 0; i < s.size(); ++i)
+        for (size_t j = i + 1; j < s.size(); ++j)
+            if (overlap(s[i].p, s[j].p, bytes))
+                return fail(err_ctx, ODSGD_ERR_OVERLAP, label(s[i]) + " overlaps " + label(s[j]));
+    return ODSGD_OK;
+}
+
+// Vector width usable for a call: 4 lanes when every pointer is 16-byte aligned, else
+// 1 lane if the context allows it.  Returns 0 and sets the error otherwise.
+int lanes_for(odsgd_ctx* c, const std::vector<Named>& ptrs) {
+    bool all16 = true;
+    for (const Named& b : ptrs) {
+        if (!aligned(b.p, 4)) {
+            fail(c, ODSGD_ERR_ALIGN, label(b) + " is not 4-byte aligned");
+            return 0;
+        }
+        if (!aligned(b.p, 16)) {
+            if (!(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED)) {
+                fail(c, ODSGD_ERR_ALIGN, label(b) + " is not 16-byte aligned (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
+                return 0;
+            }
+            all16 = false;
+        }
+    }
+    return all16 ? 4 : 1;
+}
+
+int grid_for(const odsgd_ctx* c, unsigned long long n, int lanes, int block, int per_thread, int resident_default) {
+    const unsigned long long nvec = n / lanes > 0 ? n / lanes : 1;
+    const unsigned long long tile = (unsigned long long)block * per_thread;
+    const unsigned long long tiles = (nvec + tile - 1) / tile;
+    const int per_sm = c->ctas_per_sm > 0 ? c->ctas_per_sm : resident_default;
+    const unsigned long long cap = (unsigned long long)c->sm_count * per_sm;
+    return (int)(tiles < cap ? tiles : cap);
+}
+
+int after_launch(odsgd_ctx* c, const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+    c->launches += 1;
+    return ODSGD_OK;
+}
+
+// Resident CTAs per SM for a kernel at a block size; 0 when the kernel cannot be launched
+// with that many threads (register file too small).
+template <typename K>
+int resident_ctas(K kernel, int block) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, block, 0) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = 0;
+    }
+    return n;
+}
+
+int too_wide(odsgd_ctx* c, int block) {
+    return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
+}
+
+template <bool DET, int NL, int LOCAL, int RULE>
+int launch_server_t(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    auto kernel = server_kernel<DET, NL, LOCAL, RULE>;
+    static int cached_block = 0, cached_res = 0;
+    if (cached_block != block) {
+        cached_res = resident_ctas(kernel, block);
+        cached_block = block;
+    }
+    if (cached_res == 0) return too_wide(c, block);
+    const int grid = grid_for(c, a.n, NL, block, kUnroll, cached_res);
+    kernel<<<grid, block, 0, st>>>(a);
+    return after_launch(c, "server kernel launch");
+}
+
+template <bool DET, int NL, int LOCAL>
+int launch_server_r(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+    if (LOCAL == kLocalNone) return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, st);
+    switch (c->local_rule) {
+        case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, st);
+        case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, st);
+        default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, st);
+    }
+}
+
+template <bool DET, int NL>
+int launch_server_l(odsgd_ctx* c, const ServerArgs& a, int local_mode, cudaStream_t st) {
+    switch (local_mode) {
+        case kLocalNone: return launch_server_r<DET, NL, kLocalNone>(c, a, st);
+        case kLocalOne: return launch_server_r<DET, NL, kLocalOne>(c, a, st);
+        default: return launch_server_r<DET, NL, kLocalAll>(c, a, st);
+    }
+}
+
+int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, cudaStream_t st) {
+    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    if (det) return lanes == 4 ? launch_server_l<true, 4>(c, a, local_mode, st) : launch_server_l<true, 1>(c, a, local_mode, st);
+    return lanes == 4 ? launch_server_l<false, 4>(c, a, local_mode, st) : launch_server_l<false, 1>(c, a, local_mode, st);
+}
+
+template <bool DET, int NL, int RULE>
+int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    auto kernel = local_kernel<DET, NL, RULE>;
+    static int cached_block = 0, cached_res = 0;
+    if (cached_block != block) {
+        cached_res = resident_ctas(kernel, block);
+        cached_block = block;
+    }
+    if (cached_res == 0) return too_wide(c, block);
+    kernel<<<grid_for(c, a.n, NL, block, 1, cached_res), block, 0, st>>>(a);
+    return after_launch(c, "local kernel launch");
+}
+
+template <bool DET, int NL>
+int launch_local_r(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
+    switch (c->local_rule) {
+        case ODSGD_LOCAL_SGD: return launch_local_t<DET, NL, ODSGD_LOCAL_SGD>(c, a, st);
+        case ODSGD_LOCAL_DC_C: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_C>(c, a, st);
+        default: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_A>(c, a, st);
+    }
+}
+
+int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, cudaStream_t st) {
+    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    if (det) return lanes == 4 ? launch_local_r<true, 4>(c, a, st) : launch_local_r<true, 1>(c, a, st);
+    return lanes == 4 ? launch_local_r<false, 4>(c, a, st) : launch_local_r<false, 1>(c, a, st);
+}
+
+template <bool DET, int NL>
+int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    auto kernel = asgd_kernel<DET, NL>;
+    static int cached_block = 0, cached_res = 0;
+    if (cached_block != block) {
+        cached_res = resident_ctas(kernel, block);
+        cached_block = block;
+    }
+    if (cached_res == 0) return too_wide(c, block);
+    kernel<<<grid_for(c, a.n, NL, block, 1, cached_res), block, 0, st>>>(a);
+    return after_launch(c, "asgd kernel launch");
+}
+
+int launch_asgd(odsgd_ctx* c, const AsgdArgs& a, int lanes, cudaStream_t st) {
+    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    if (det) return lanes == 4 ? launch_asgd_t<true, 4>(c, a, st) : launch_asgd_t<true, 1>(c, a, st);
+    return lanes == 4 ? launch_asgd_t<false, 4>(c, a, st) : launch_asgd_t<false, 1>(c, a, st);
+}
+
+LocalParams local_params(const odsgd_ctx* c) {
+    LocalParams p;
+    p.local_lr = c->local_lr;
+    p.lambda = c->dc_lambda;
+    p.m = c->dc_m;
+    p.one_minus_m = 1.0f - c->dc_m;
+    p.eps = c->dc_eps;
+    return p;
+}
+
+// Checks a table of gradient pointers against the context's state buffers.
+int check_grads(odsgd_ctx* c, const float* const* grads, std::vector<Named>* ptrs) {
+    if (!grads) return fail(c, ODSGD_ERR_ARG, "worker_grads is NULL");
+    const size_t bytes = c->n * sizeof(float);
+    const std::vector<Named> st = state_buffers(c);
+    for (int m = 0; m < c->n_workers; ++m) {
+        if (!grads[m]) return fail(c, ODSGD_ERR_ARG, "worker_grads[" + std::to_string(m) + "] is NULL");
+        const Named g{grads[m], "worker_grads", m};
+        for (const Named& s : st)
+            if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, label(g) + " overlaps " + label(s));
+        ptrs->push_back(g);
+    }
+    return ODSGD_OK;
+}
+
+// Local mode and outputs for a fused call; fills a.x / a.ms / a.local_worker.
+int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mode, std::vector<Named>* ptrs) {
+    if (worker_id >= c->n_workers || worker_id < -1) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
+    if (worker_id >= 0) {
+        if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
+        if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for that worker");
+        a->x[0] = c->local[worker_id];
+        a->ms[0] = c->mean_square[worker_id];
+        a->local_worker = worker_id;
+        ptrs->push_back({a->x[0], "local", worker_id});
+        if (need_ms) ptrs->push_back({a->ms[0], "mean_square", worker_id});
+        *local_mode = kLocalOne;
+        return ODSGD_OK;
+    }
+    int count = 0;
+    for (int m = 0; m < c->n_workers; ++m) {
+        a->x[m] = c->local[m];
+        a->ms[m] = c->mean_square[m];
+        if (c->local[m]) {
+            if (need_ms && !c->mean_square[m]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for worker " + std::to_string(m));
+            ptrs->push_back({a->x[m], "local", m});
+            if (need_ms) ptrs->push_back({a->ms[m], "mean_square", m});
+            ++count;
+        }
+    }
+    if (count == 0) return fail(c, ODSGD_ERR_ARG, "worker_id == -1 but the context has no local buffers");
+    *local_mode = kLocalAll;
+    return ODSGD_OK;
+}
+
+// Shared body of the global, fused and SSGD calls.
+//   keep_backup: OD-SGD server step (the old weights stay available to the workers)
+//   local_id:    -2 none, -1 all workers, >= 0 one worker
+int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, void* stream) {
+    if (!c) return ODSGD_ERR_ARG;
+    std::vector<Named> ptrs;
+    int rc = check_grads(c, grads, &ptrs);
+    if (rc != ODSGD_OK) return rc;
+
+    ServerArgs a;
+    memset(&a, 0, sizeof a);
+    for (int m = 0; m < c->n_workers; ++m) a.g[m] = grads[m];
+    a.v = c->v;
+    a.n = c->n;
+    a.n_workers = c->n_workers;
+    a.inv_n = 1.0f / (float)c->n_workers;
+    a.lr = c->lr;
+    a.momentum = c->momentum;
+    a.wd = c->wd;
+    a.lp = local_params(c);
+    a.w_in = c->w[c->cur];
+    const float* delayed_after = nullptr;
+    int next_cur = c->cur;
+    if (keep_backup && c->pingpong) {
+        a.w_out = c->w[c->cur ^ 1];
+        delayed_after = c->w[c->cur];
+        next_cur = c->cur ^ 1;
+    } else {
+        a.w_out = c->w[c->cur];
+        if (keep_backup && c->w_delayed) {
+            a.w_prev = c->w_delayed;
+            delayed_after = c->w_delayed;
+        }
+    }
+    ptrs.push_back({a.w_in, "w", -1});
+    ptrs.push_back({a.w_out, "w", -1});
+    ptrs.push_back({a.v, "v", -1});
+    if (a.w_prev) ptrs.push_back({a.w_prev, "w_delayed", -1});
+
+    int local_mode = kLocalNone;
+    if (local_id >= -1) {
+        rc = bind_local_outputs(c, local_id, &a, &local_mode, &ptrs);
+        if (rc != ODSGD_OK) return rc;
+    }
+    const int lanes = lanes_for(c, ptrs);
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+
+    rc = launch_server(c, a, lanes, local_mode, static_cast<cudaStream_t>(stream));
+    if (rc != ODSGD_OK) return rc;
+
+    c->cur = next_cur;
+    c->step += 1;
+    c->delayed = delayed_after;
+    c->grads_bound = keep_backup;
+    if (keep_backup)
+        for (int m = 0; m < c->n_workers; ++m) c->bound[m] = grads[m];
+    return ODSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int odsgd_version(void) { return ODSGD_VERSION_MAJOR * 1000 + ODSGD_VERSION_MINOR; }
+
+const char* odsgd_strerror(int code) {
+    switch (code) {
+        case ODSGD_OK: return "ok";
+        case ODSGD_ERR_ARG: return "invalid argument";
+        case ODSGD_ERR_ALIGN: return "misaligned device pointer";
+        case ODSGD_ERR_OVERLAP: return "buffers overlap";
+        case ODSGD_ERR_STATE: return "call not valid in this state";
+        case ODSGD_ERR_CUDA: return "CUDA error";
+        case ODSGD_ERR_UNSUPPORTED: return "not supported";
+        default: return "unknown error code";
+    }
+}
+
+int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
+    if (!out) return fail(nullptr, ODSGD_ERR_ARG, "out is NULL");
+    *out = nullptr;
+    if (!d) return fail(nullptr, ODSGD_ERR_ARG, "desc is NULL");
+    if (!d->w_a || !d->v) return fail(nullptr, ODSGD_ERR_ARG, "w_a and v must not be NULL");
+    if (d->n_params == 0) return fail(nullptr, ODSGD_ERR_ARG, "n_params is 0");
+    if (d->n_workers < 1 || d->n_workers > ODSGD_MAX_WORKERS)
+        return fail(nullptr, ODSGD_ERR_ARG, "n_workers must be in 1.." + std::to_string(ODSGD_MAX_WORKERS));
+    if (d->w_b && d->w_delayed) return fail(nullptr, ODSGD_ERR_ARG, "w_delayed must be NULL in the ping-pong layout");
+    if (!d->tensor_offsets || d->n_tensors < 1) return fail(nullptr, ODSGD_ERR_ARG, "tensor_offsets / n_tensors missing");
+    if (d->tensor_offsets[0] != 0 || d->tensor_offsets[d->n_tensors] != d->n_params)
+        return fail(nullptr, ODSGD_ERR_ARG, "tensor_offsets must start at 0 and end at n_params");
+    for (size_t t = 0; t < d->n_tensors; ++t)
+        if (d->tensor_offsets[t + 1] <= d->tensor_offsets[t])
+            return fail(nullptr, ODSGD_ERR_ARG, "tensor_offsets must be strictly ascending (at tensor " + std::to_string(t) + ")");
+    if (d->flags & ~(ODSGD_FLAG_DETERMINISTIC | ODSGD_FLAG_ALLOW_UNALIGNED))
+        return fail(nullptr, ODSGD_ERR_ARG, "unknown flag bits");
+
+    odsgd_ctx* c = new (std::nothrow) odsgd_ctx;
+    if (!c) return fail(nullptr, ODSGD_ERR_ARG, "out of host memory");
+    c->w[0] = d->w_a;
+    c->w[1] = d->w_b;
+    c->pingpong = d->w_b != nullptr;
+    c->w_delayed = d->w_delayed;
+    c->v = d->v;
+    c->n = d->n_params;
+    c->n_workers = d->n_workers;
+    c->offsets.assign(d->tensor_offsets, d->tensor_offsets + d->n_tensors + 1);
+    c->lr = d->lr;
+    c->local_lr = d->local_lr;
+    c->momentum = d->momentum;
+    c->wd = d->wd;
+    c->flags = d->flags;
+    if (d->local)
+        for (int m = 0; m < d->n_workers; ++m) c->local[m] = d->local[m];
+
+    const std::vector<Named> st = state_buffers(c);
+    const size_t need = (d->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
+    for (const Named& b : st) {
+        if (!aligned(b.p, need)) {
+            const std::string msg = label(b) + " is not " + std::to_string(need) + "-byte aligned";
+            delete c;
+            return fail(nullptr, ODSGD_ERR_ALIGN, msg);
+        }
+    }
+    int rc = check_distinct(nullptr, st, c->n * sizeof(float));
+    if (rc != ODSGD_OK) {
+        delete c;
+        return rc;
+    }
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess || c->sm_count < 1) {
+        const std::string msg = std::string("no usable CUDA device: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        delete c;
+        return fail(nullptr, ODSGD_ERR_CUDA, msg);
+    }
+    *out = c;
+    return ODSGD_OK;
+}
+
+int odsgd_destroy(odsgd_ctx* ctx) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    delete ctx;
+    return ODSGD_OK;
+}
+
+int odsgd_global_update(odsgd_ctx* ctx, const float* const* worker_grads, void* stream) {
+    return server_call(ctx, worker_grads, true, -2, stream);
+}
+
+int odsgd_fused_update(odsgd_ctx* ctx, const float* const* worker_grads, int worker_id, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (worker_id < -1 || worker_id >= ctx->n_workers) return fail(ctx, ODSGD_ERR_ARG, "worker_id out of range");
+    return server_call(ctx, worker_grads, true, worker_id, stream);
+}
+
+int odsgd_ssgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream) {
+    return server_call(ctx, worker_grads, false, -2, stream);
+}
+
+int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (!c->grads_bound) return fail(c, ODSGD_ERR_STATE, "no gradients bound: call odsgd_global_update first");
+    if (!c->delayed) return fail(c, ODSGD_ERR_STATE, "this context keeps no backup weights (in-place layout without w_delayed)");
+    if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
+    const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
+    if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for that worker");
+    LocalArgs a;
+    a.w_bak = c->delayed;
+    a.g = c->bound[worker_id];
+    a.x = c->local[worker_id];
+    a.ms = c->mean_square[worker_id];
+    a.n = c->n;
+    a.lp = local_params(c);
+    std::vector<Named> ptrs = {{a.w_bak, "w_delayed", -1}, {a.g, "worker_grads", worker_id}, {a.x, "local", worker_id}};
+    if (need_ms) ptrs.push_back({a.ms, "mean_square", worker_id});
+    const int lanes = lanes_for(c, ptrs);
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+    return launch_local(c, a, lanes, static_cast<cudaStream_t>(stream));
+}
+
+int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging, int worker_id,
+                            float* host_local_out, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (!host_grads || !dev_staging) return fail(c, ODSGD_ERR_ARG, "host_grads / dev_staging is NULL");
+    if (worker_id < -1 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (host_local_out && worker_id < 0) return fail(c, ODSGD_ERR_ARG, "host_local_out needs worker_id >= 0");
+    for (int m = 0; m < c->n_workers; ++m)
+        if (!host_grads[m] || !dev_staging[m]) return fail(c, ODSGD_ERR_ARG, "NULL entry in host_grads / dev_staging");
+    // validate before the first copy is enqueued
+    std::vector<Named> ptrs;
+    int rc = check_grads(c, dev_staging, &ptrs);
+    if (rc != ODSGD_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t bytes = c->n * sizeof(float);
+    for (int m = 0; m < c->n_workers; ++m) {
+        const cudaError_t e = cudaMemcpyAsync(dev_staging[m], host_grads[m], bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("host-to-device copy: ") + cudaGetErrorString(e));
+    }
+    rc = server_call(c, dev_staging, true, worker_id, stream);
+    if (rc != ODSGD_OK) return rc;
+    if (host_local_out) {
+        const cudaError_t e = cudaMemcpyAsync(host_local_out, c->local[worker_id], bytes, cudaMemcpyDeviceToHost, st);
+        if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("device-to-host copy: ") + cudaGetErrorString(e));
+    }
+    return ODSGD_OK;
+}
+
+int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (!grad) return fail(c, ODSGD_ERR_ARG, "grad is NULL");
+    const size_t bytes = c->n * sizeof(float);
+    const Named g{grad, "grad", -1};
+    for (const Named& s : state_buffers(c))
+        if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, "grad overlaps " + label(s));
+    AsgdArgs a;
+    a.g = grad;
+    a.w = c->w[c->cur];
+    a.v = c->v;
+    a.n = c->n;
+    a.lr = c->lr;
+    a.momentum = c->momentum;
+    a.wd = c->wd;
+    const int lanes = lanes_for(c, {g, {a.w, "w", -1}, {a.v, "v", -1}});
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+    const int rc = launch_asgd(c, a, lanes, static_cast<cudaStream_t>(stream));
+    if (rc != ODSGD_OK) return rc;
+    c->step += 1;
+    c->grads_bound = false;
+    c->delayed = nullptr;
+    return ODSGD_OK;
+}
+
+int odsgd_set_lr(odsgd_ctx* ctx, float lr) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->lr = lr;
+    return ODSGD_OK;
+}
+
+int odsgd_set_local_lr(odsgd_ctx* ctx, float local_lr) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->local_lr = local_lr;
+    return ODSGD_OK;
+}
+
+int odsgd_set_momentum(odsgd_ctx* ctx, float momentum) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->momentum = momentum;
+    return ODSGD_OK;
+}
+
+int odsgd_set_wd(odsgd_ctx* ctx, float wd) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->wd = wd;
+    return ODSGD_OK;
+}
+
+int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float eps, float* const* mean_square) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (rule != ODSGD_LOCAL_SGD && rule != ODSGD_LOCAL_DC_C && rule != ODSGD_LOCAL_DC_A)
+        return fail(c, ODSGD_ERR_ARG, "unknown local rule");
+    if (rule == ODSGD_LOCAL_DC_A) {
+        if (!mean_square) return fail(c, ODSGD_ERR_ARG, "ODSGD_LOCAL_DC_A needs mean_square arenas");
+        odsgd_ctx probe = *c;
+        for (int w = 0; w < c->n_workers; ++w) probe.mean_square[w] = mean_square[w];
+        const std::vector<Named> st = state_buffers(&probe);
+        const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
+        for (int w = 0; w < c->n_workers; ++w) {
+            if (c->local[w] && !mean_square[w]) return fail(c, ODSGD_ERR_ARG, "mean_square[" + std::to_string(w) + "] is NULL");
+            if (mean_square[w] && !aligned(mean_square[w], need)) return fail(c, ODSGD_ERR_ALIGN, "mean_square arena misaligned");
+        }
+        const int rc = check_distinct(c, st, c->n * sizeof(float));
+        if (rc != ODSGD_OK) return rc;
+        for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = mean_square[w];
+    } else {
+        for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = nullptr;
+    }
+    c->local_rule = rule;
+    c->dc_lambda = lambda;
+    c->dc_m = m;
+    c->dc_eps = eps;
+    return ODSGD_OK;
+}
+
+int odsgd_get_weights(odsgd_ctx* ctx, float** current, float** delayed) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (current) *current = ctx->w[ctx->cur];
+    if (delayed) *delayed = const_cast<float*>(ctx->delayed);
+    return ODSGD_OK;
+}
+
+int odsgd_get_step(odsgd_ctx* ctx, uint64_t* step) {
+    if (!ctx || !step) return ODSGD_ERR_ARG;
+    *step = ctx->step;
+    return ODSGD_OK;
+}
+
+int odsgd_set_step(odsgd_ctx* ctx, uint64_t step) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->step = step;
+    return ODSGD_OK;
+}
+
+int odsgd_set_launch_config(odsgd_ctx* ctx, int block_threads, int ctas_per_sm) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (block_threads != 0 && (block_threads < 64 || block_threads > 1024 || block_threads % 32 != 0))
+        return fail(ctx, ODSGD_ERR_ARG, "block_threads must be 0 or a multiple of 32 in 64..1024");
+    if (ctas_per_sm < 0) return fail(ctx, ODSGD_ERR_ARG, "ctas_per_sm must be >= 0");
+    ctx->block_threads = block_threads;
+    ctx->ctas_per_sm = ctas_per_sm;
+    return ODSGD_OK;
+}
+
+int odsgd_get_launch_count(odsgd_ctx* ctx, uint64_t* launches) {
+    if (!ctx || !launches) return ODSGD_ERR_ARG;
+    *launches = ctx->launches;
+    return ODSGD_OK;
+}
+
+const char* odsgd_last_error(odsgd_ctx* ctx) {
+    return ctx ? ctx->err.c_str() : g_create_err.c_str();
+}
+
+}  // extern "C"

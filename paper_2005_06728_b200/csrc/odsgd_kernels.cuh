@@ -1,0 +1,323 @@
+// Device code of the OD-SGD update pass for sm_100a.
+//
+// All rules are element-wise and bound by HBM bandwidth (about a quarter of a
+// flop per byte), so the kernels are organised around memory traffic only:
+//   * every input stream is read exactly once and every output written once;
+//   * 128-bit loads and stores, each warp touching 512 contiguous bytes per
+//     stream per instruction, each CTA walking contiguous tiles of every stream;
+//   * the M gradient streams are fetched in batches of kBatch independent
+//     loads per thread before the dependent adds start, which keeps tens of KB
+//     in flight per SM; the adds themselves stay in worker order 0..M-1;
+//   * read-once data is loaded with the streaming policy and results are
+//     stored with the streaming policy, so nothing useful is pushed out of L2;
+//   * a persistent grid (SMs x resident CTAs) strides over the tiles, so one
+//     launch covers the whole arena whatever the number of tensors in it.
+// Tensor cores have no role here: there is no contraction.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "odsgd.h"
+
+namespace odsgd {
+
+#ifndef ODSGD_BATCH
+#define ODSGD_BATCH 8  // gradient loads in flight per thread and vector
+#endif
+#ifndef ODSGD_UNROLL
+#define ODSGD_UNROLL 1  // vectors per thread per tile
+#endif
+constexpr int kBatch = ODSGD_BATCH;
+constexpr int kUnroll = ODSGD_UNROLL;
+
+enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
+
+struct LocalParams {
+    float local_lr;
+    float lambda;       // Eq. 4 / Eq. 5 compensation coefficient
+    float m;            // Eq. 6 decay
+    float one_minus_m;  // computed once on the host in fp32
+    float eps;          // Eq. 5
+};
+
+// Kernel argument block, passed by value (constant bank): no dependent device
+// load is needed to find a worker's gradient buffer.
+struct ServerArgs {
+    const float* g[ODSGD_MAX_WORKERS];  // gradient arenas, worker order
+    float* x[ODSGD_MAX_WORKERS];        // local-weight arenas (kLocalAll) or x[0] (kLocalOne)
+    float* ms[ODSGD_MAX_WORKERS];       // Eq. 6 state, same indexing as x
+    const float* w_in;                  // weights before the update
+    float* w_out;                       // weights after the update (may equal w_in)
+    float* w_prev;                      // optional copy of the old weights
+    float* v;                           // momentum state, in place
+    unsigned long long n;               // elements
+    int n_workers;
+    int local_worker;                   // kLocalOne: whose gradient feeds x[0]
+    float inv_n;                        // 1.0f / n_workers, computed on the host
+    float lr, momentum, wd;
+    LocalParams lp;
+};
+
+struct LocalArgs {
+    const float* w_bak;
+    const float* g;
+    float* x;   // read (previous local weights) by the delay-compensated rules, then written
+    float* ms;  // Eq. 6 state or null
+    unsigned long long n;
+    LocalParams lp;
+};
+
+struct AsgdArgs {
+    const float* g;
+    float* w;
+    float* v;
+    unsigned long long n;
+    float lr, momentum, wd;
+};
+
+// ------------------------------------------------------------------ vectors
+template <int NL>
+struct Vec {
+    float e[NL];
+};
+
+template <int NL>
+__device__ __forceinline__ Vec<NL> load_stream(const float* p);
+template <>
+__device__ __forceinline__ Vec<4> load_stream<4>(const float* p) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+    return Vec<4>{{t.x, t.y, t.z, t.w}};
+}
+template <>
+__device__ __forceinline__ Vec<1> load_stream<1>(const float* p) {
+    return Vec<1>{{__ldcs(p)}};
+}
+
+template <int NL>
+__device__ __forceinline__ void store_stream(float* p, const Vec<NL>& a);
+template <>
+__device__ __forceinline__ void store_stream<4>(float* p, const Vec<4>& a) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(a.e[0], a.e[1], a.e[2], a.e[3]));
+}
+template <>
+__device__ __forceinline__ void store_stream<1>(float* p, const Vec<1>& a) {
+    __stcs(p, a.e[0]);
+}
+
+// ------------------------------------------------------------------ arithmetic
+// DET: each operator is its own correctly rounded binary32 operation (the
+// intrinsics are never contracted).  Otherwise plain operators, which the
+// compiler may contract into fused multiply-adds.
+template <bool DET>
+struct Op {
+    static __device__ __forceinline__ float add(float a, float b) { return DET ? __fadd_rn(a, b) : a + b; }
+    static __device__ __forceinline__ float sub(float a, float b) { return DET ? __fsub_rn(a, b) : a - b; }
+    static __device__ __forceinline__ float mul(float a, float b) { return DET ? __fmul_rn(a, b) : a * b; }
+    static __device__ __forceinline__ float div(float a, float b) { return DET ? __fdiv_rn(a, b) : a / b; }
+    static __device__ __forceinline__ float sqrt(float a) { return DET ? __fsqrt_rn(a) : sqrtf(a); }
+};
+
+// Momentum SGD with L2 decay on one element (Algorithm 1's "Update w_t").
+template <bool DET>
+__device__ __forceinline__ void server_rule(float gbar, float w, float v, float lr, float momentum, float wd,
+                                            float& w_new, float& v_new) {
+    using O = Op<DET>;
+    const float d = O::add(gbar, O::mul(wd, w));
+    v_new = O::sub(O::mul(momentum, v), O::mul(lr, d));
+    w_new = O::add(w, v_new);
+}
+
+// Local updater on one element (Section 3.3).  x_prev / ms are only touched by
+// the delay-compensated rules.
+template <bool DET, int RULE>
+__device__ __forceinline__ float local_rule(float w_bak, float g, float x_prev, float& ms, const LocalParams& p) {
+    using O = Op<DET>;
+    if (RULE == ODSGD_LOCAL_SGD) {
+        return O::sub(w_bak, O::mul(p.local_lr, g));
+    }
+    const float gg = O::mul(g, g);
+    float lam = p.lambda;
+    if (RULE == ODSGD_LOCAL_DC_A) {
+        ms = O::add(O::mul(p.m, ms), O::mul(p.one_minus_m, gg));  // Eq. 6
+        lam = O::div(p.lambda, O::sqrt(O::add(ms, p.eps)));
+    }
+    const float diff = O::sub(w_bak, x_prev);
+    const float comp = O::mul(O::mul(lam, gg), diff);
+    return O::sub(w_bak, O::mul(p.local_lr, O::add(g, comp)));  // Eq. 4 / Eq. 5
+}
+
+// ------------------------------------------------------------------ server kernel
+// One vector (NL lanes) of the arena at element offset `off`:
+// sum the workers in order, apply the server rule, and (LOCAL != none) the
+// local rule for one worker or for every worker that has a local buffer.
+template <bool DET, int NL, int LOCAL, int RULE, int U>
+__device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsigned long long (&off)[U],
+                                               const bool (&ok)[U]) {
+    using O = Op<DET>;
+    Vec<NL> w[U], v[U], s[U], gl[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (ok[u]) {
+            w[u] = load_stream<NL>(a.w_in + off[u]);
+            v[u] = load_stream<NL>(a.v + off[u]);
+        }
+    }
+    const int n_workers = a.n_workers;
+    for (int m0 = 0; m0 < n_workers; m0 += kBatch) {
+        Vec<NL> t[kBatch][U];
+        // independent loads first ...
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            if (m0 + j < n_workers) {
+                const float* gp = a.g[m0 + j];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (ok[u]) t[j][u] = load_stream<NL>(gp + off[u]);
+                }
+            }
+        }
+        // ... then the adds, strictly in worker order
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            const int m = m0 + j;
+            if (m < n_workers) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (ok[u]) {
+                        if (m == 0) {
+                            s[u] = t[j][u];
+                        } else {
+#pragma unroll
+                            for (int l = 0; l < NL; ++l) s[u].e[l] = O::add(s[u].e[l], t[j][u].e[l]);
+                        }
+                        if (LOCAL == kLocalOne) {
+                            if (m == a.local_worker) gl[u] = t[j][u];
+                        }
+                        if (LOCAL == kLocalAll) {
+                            float* xp = a.x[m];
+                            if (xp != nullptr) {
+                                Vec<NL> xo, xv, msv;
+                                if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(xp + off[u]);
+                                if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[m] + off[u]);
+#pragma unroll
+                                for (int l = 0; l < NL; ++l) {
+                                    xo.e[l] = local_rule<DET, RULE>(w[u].e[l], t[j][u].e[l], xv.e[l], msv.e[l], a.lp);
+                                }
+                                store_stream<NL>(xp + off[u], xo);
+                                if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[m] + off[u], msv);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        Vec<NL> wn, vn;
+#pragma unroll
+        for (int l = 0; l < NL; ++l) {
+            const float gbar = O::mul(s[u].e[l], a.inv_n);
+            server_rule<DET>(gbar, w[u].e[l], v[u].e[l], a.lr, a.momentum, a.wd, wn.e[l], vn.e[l]);
+        }
+        if (LOCAL == kLocalOne) {
+            float* xp = a.x[0];
+            Vec<NL> xo, xv, msv;
+            if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(xp + off[u]);
+            if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[0] + off[u]);
+#pragma unroll
+            for (int l = 0; l < NL; ++l) {
+                xo.e[l] = local_rule<DET, RULE>(w[u].e[l], gl[u].e[l], xv.e[l], msv.e[l], a.lp);
+            }
+            store_stream<NL>(xp + off[u], xo);
+            if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[0] + off[u], msv);
+        }
+        if (a.w_prev != nullptr) store_stream<NL>(a.w_prev + off[u], w[u]);
+        store_stream<NL>(a.v + off[u], vn);
+        store_stream<NL>(a.w_out + off[u], wn);
+    }
+}
+
+template <bool DET, int NL, int LOCAL, int RULE>
+__global__ void server_kernel(const __grid_constant__ ServerArgs a) {
+    const unsigned long long nvec = a.n / NL;
+    const unsigned long long tile = (unsigned long long)blockDim.x * kUnroll;
+    const unsigned long long stride = (unsigned long long)gridDim.x * tile;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * tile; base < nvec; base += stride) {
+        unsigned long long off[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const unsigned long long i = base + (unsigned long long)u * blockDim.x + threadIdx.x;
+            ok[u] = i < nvec;
+            off[u] = i * NL;
+        }
+        server_vectors<DET, NL, LOCAL, RULE, kUnroll>(a, off, ok);
+    }
+    if (NL > 1) {
+        // ragged tail: the last n % NL elements, one lane each
+        const unsigned long long done = nvec * NL;
+        if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
+            const unsigned long long off1[1] = {done + threadIdx.x};
+            const bool ok1[1] = {true};
+            server_vectors<DET, 1, LOCAL, RULE, 1>(a, off1, ok1);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ local kernel
+template <bool DET, int NL, int RULE>
+__device__ __forceinline__ void local_vector(const LocalArgs& a, unsigned long long off) {
+    const Vec<NL> w = load_stream<NL>(a.w_bak + off);
+    const Vec<NL> g = load_stream<NL>(a.g + off);
+    Vec<NL> xv, msv, xo;
+    if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(a.x + off);
+    if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms + off);
+#pragma unroll
+    for (int l = 0; l < NL; ++l) xo.e[l] = local_rule<DET, RULE>(w.e[l], g.e[l], xv.e[l], msv.e[l], a.lp);
+    store_stream<NL>(a.x + off, xo);
+    if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms + off, msv);
+}
+
+template <bool DET, int NL, int RULE>
+__global__ void local_kernel(const __grid_constant__ LocalArgs a) {
+    const unsigned long long nvec = a.n / NL;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        local_vector<DET, NL, RULE>(a, i * NL);
+    }
+    if (NL > 1) {
+        const unsigned long long done = nvec * NL;
+        if (blockIdx.x == 0 && done + threadIdx.x < a.n) local_vector<DET, 1, RULE>(a, done + threadIdx.x);
+    }
+}
+
+// ------------------------------------------------------------------ ASGD kernel
+template <bool DET, int NL>
+__device__ __forceinline__ void asgd_vector(const AsgdArgs& a, unsigned long long off) {
+    const Vec<NL> g = load_stream<NL>(a.g + off);
+    const Vec<NL> w = load_stream<NL>(a.w + off);
+    const Vec<NL> v = load_stream<NL>(a.v + off);
+    Vec<NL> wn, vn;
+#pragma unroll
+    for (int l = 0; l < NL; ++l) server_rule<DET>(g.e[l], w.e[l], v.e[l], a.lr, a.momentum, a.wd, wn.e[l], vn.e[l]);
+    store_stream<NL>(a.v + off, vn);
+    store_stream<NL>(a.w + off, wn);
+}
+
+template <bool DET, int NL>
+__global__ void asgd_kernel(const __grid_constant__ AsgdArgs a) {
+    const unsigned long long nvec = a.n / NL;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
+        asgd_vector<DET, NL>(a, i * NL);
+    }
+    if (NL > 1) {
+        const unsigned long long done = nvec * NL;
+        if (blockIdx.x == 0 && done + threadIdx.x < a.n) asgd_vector<DET, 1>(a, done + threadIdx.x);
+    }
+}
+
+}  // namespace odsgd

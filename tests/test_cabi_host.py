@@ -1,0 +1,148 @@
+"""The C-ABI library loads without a GPU, exports everything the header declares, and its
+argument checks answer before any CUDA call is made.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2005_06728_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()  # no-op when the in-tree library is up to date
+    return binding.load_library()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "odsgd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(odsgd_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared()
+    assert len(names) >= 20
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in odsgd.h but missing from libodsgd.so"
+    assert sorted(binding.EXPORTS) == names, "binding.EXPORTS must list exactly the header's entry points"
+
+
+def test_version_and_strerror(lib):
+    assert lib.odsgd_version() == 1
+    assert lib.odsgd_strerror(0) == b"ok"
+    assert b"overlap" in lib.odsgd_strerror(binding.ERR_OVERLAP)
+    assert b"unknown" in lib.odsgd_strerror(-99)
+
+
+def _desc(**over):
+    n = 1024
+    offs = (ctypes.c_size_t * 3)(0, 512, n)
+    d = binding._Desc()
+    d.w_a, d.v = 0x10000, 0x20000  # never dereferenced: create() only inspects the values
+    d.n_params, d.n_tensors, d.n_workers = n, 2, 4
+    d.tensor_offsets = ctypes.cast(offs, ctypes.POINTER(ctypes.c_size_t))
+    d.lr, d.local_lr, d.momentum, d.wd, d.flags = 0.1, 0.1, 0.9, 0.0, 0
+    d._keep = offs
+    for k, val in over.items():
+        setattr(d, k, val)
+    return d
+
+
+def _create(lib, d):
+    h = ctypes.c_void_p(1)
+    rc = lib.odsgd_create(ctypes.byref(h), ctypes.byref(d))
+    return rc, h, lib.odsgd_last_error(None).decode()
+
+
+@pytest.mark.parametrize("over,code,word", [
+    (dict(w_a=None), binding.ERR_ARG, "NULL"),
+    (dict(v=None), binding.ERR_ARG, "NULL"),
+    (dict(n_params=0), binding.ERR_ARG, "n_params"),
+    (dict(n_workers=0), binding.ERR_ARG, "n_workers"),
+    (dict(n_workers=binding.MAX_WORKERS + 1), binding.ERR_ARG, "n_workers"),
+    (dict(w_b=0x30000, w_delayed=0x40000), binding.ERR_ARG, "w_delayed"),
+    (dict(n_tensors=0), binding.ERR_ARG, "tensor_offsets"),
+    (dict(flags=0x80), binding.ERR_ARG, "flag"),
+    (dict(w_a=0x10004), binding.ERR_ALIGN, "w_a"),
+    (dict(v=0x10000 + 4 * 1000), binding.ERR_OVERLAP, "overlaps"),
+    (dict(w_b=0x20000 + 16), binding.ERR_OVERLAP, "overlaps"),
+])
+def test_create_rejects_bad_descriptions(lib, over, code, word):
+    rc, h, msg = _create(lib, _desc(**over))
+    assert rc == code, msg
+    assert h.value is None, "*out must be NULL on failure"
+    assert word in msg
+
+
+def test_create_checks_offsets(lib):
+    d = _desc()
+    bad = (ctypes.c_size_t * 3)(0, 512, 1000)  # does not end at n_params
+    d.tensor_offsets = ctypes.cast(bad, ctypes.POINTER(ctypes.c_size_t))
+    assert _create(lib, d)[0] == binding.ERR_ARG
+    bad2 = (ctypes.c_size_t * 3)(0, 0, 1024)  # empty tensor
+    d.tensor_offsets = ctypes.cast(bad2, ctypes.POINTER(ctypes.c_size_t))
+    rc, _, msg = _create(lib, d)
+    assert rc == binding.ERR_ARG and "ascending" in msg
+    bad3 = (ctypes.c_size_t * 3)(4, 512, 1024)
+    d.tensor_offsets = ctypes.cast(bad3, ctypes.POINTER(ctypes.c_size_t))
+    assert _create(lib, d)[0] == binding.ERR_ARG
+
+
+def test_unaligned_flag_relaxes_alignment_only_to_four_bytes(lib):
+    import torch
+
+    rc, _, msg = _create(lib, _desc(w_a=0x10004, flags=binding.FLAG_ALLOW_UNALIGNED))
+    if torch.cuda.is_available():
+        assert rc == binding.OK
+    else:
+        assert rc == binding.ERR_CUDA, "a valid description gets as far as the device query"
+    rc, _, msg = _create(lib, _desc(w_a=0x10002, flags=binding.FLAG_ALLOW_UNALIGNED))
+    assert rc == binding.ERR_ALIGN
+
+
+def test_local_table_is_checked(lib):
+    tab = (ctypes.c_void_p * 4)(0x50000, None, 0x50000 + 64, None)  # two locals overlap
+    d = _desc()
+    d.local = ctypes.cast(tab, ctypes.POINTER(ctypes.c_void_p))
+    rc, _, msg = _create(lib, d)
+    assert rc == binding.ERR_OVERLAP and "local[0]" in msg and "local[2]" in msg
+
+
+def test_null_context_is_an_argument_error(lib):
+    null = ctypes.c_void_p()
+    assert lib.odsgd_destroy(null) == binding.ERR_ARG
+    assert lib.odsgd_global_update(null, None, None) == binding.ERR_ARG
+    assert lib.odsgd_local_update(null, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_fused_update(null, None, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_fused_update_host(null, None, None, 0, None, None) == binding.ERR_ARG
+    assert lib.odsgd_ssgd_step(null, None, None) == binding.ERR_ARG
+    assert lib.odsgd_asgd_step(null, 0, None, None) == binding.ERR_ARG
+    assert lib.odsgd_set_lr(null, 0.1) == binding.ERR_ARG
+    assert lib.odsgd_set_launch_config(null, 256, 1) == binding.ERR_ARG
+    assert lib.odsgd_get_step(null, None) == binding.ERR_ARG
+    assert lib.odsgd_create(None, None) == binding.ERR_ARG
+    assert lib.odsgd_last_error(null) is not None
+
+
+def test_missing_library_fails_loudly(tmp_path):
+    with pytest.raises(RuntimeError, match="no fallback"):
+        binding.load_library(str(tmp_path / "libodsgd.so"))
+
+
+def test_product_does_not_reach_for_the_oracle():
+    """Nothing in the package imports, loads or calls the oracle (the reverse holds too)."""
+    pkg = os.path.join(ROOT, "paper_2005_06728_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(import|from)\s+oracle\b", text, re.M), f"{f} imports the oracle"
+                assert "odsgd_oracle" not in text and "oracle/" not in text and "oracle_" not in text, f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".cpp", ".h")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2005_06728_b200" not in text and "odsgd.h" not in text
