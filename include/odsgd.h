@@ -216,9 +216,10 @@ int odsgd_get_step(odsgd_ctx* ctx, uint64_t* step);
 int odsgd_set_step(odsgd_ctx* ctx, uint64_t step);
 
 /*
- * Launch shape of the update kernels.  block_threads: 64..1024, multiple of 32;
- * ctas_per_sm: >= 1, grid = min(tiles, SMs * ctas_per_sm) persistent CTAs; 0 for
- * either restores the built-in choice.
+ * Launch shape of the update kernels.  block_threads: 64..1024, multiple of 32 (a block
+ * too large for a kernel's register use makes that call fail with ERR_UNSUPPORTED);
+ * ctas_per_sm: >= 1, grid = min(tiles, SMs * ctas_per_sm) CTAs striding over the tiles;
+ * 0 for either restores the built-in choice.
  */
 int odsgd_set_launch_config(odsgd_ctx* ctx, int block_threads, int ctas_per_sm);
 

@@ -5,13 +5,17 @@
 //   * every input stream is read exactly once and every output written once;
 //   * 128-bit loads and stores, each warp touching 512 contiguous bytes per
 //     stream per instruction, each CTA walking contiguous tiles of every stream;
-//   * the M gradient streams are fetched in batches of kBatch independent
-//     loads per thread before the dependent adds start, which keeps tens of KB
-//     in flight per SM; the adds themselves stay in worker order 0..M-1;
-//   * read-once data is loaded with the streaming policy and results are
-//     stored with the streaming policy, so nothing useful is pushed out of L2;
-//   * a persistent grid (SMs x resident CTAs) strides over the tiles, so one
-//     launch covers the whole arena whatever the number of tensors in it.
+//   * the M gradient streams are fetched in batches of kBatch x kUnroll
+//     independent 128-bit loads per thread before the dependent adds start
+//     (about 160 KB in flight per SM at two resident CTAs); the adds themselves
+//     stay in worker order 0..M-1;
+//   * gradients go through the read-only path (ld.global.nc), which measured
+//     5-8 % faster here than streaming loads (ld.global.cs); state that is read
+//     and written by the same kernel uses coherent loads; results are stored
+//     with the streaming policy;
+//   * a grid of SMs x 64 CTAs at most strides over the tiles, so one launch
+//     covers the whole arena whatever the number of tensors in it, and the
+//     hardware scheduler evens out the tail.
 // Tensor cores have no role here: there is no contraction.
 #pragma once
 
@@ -26,10 +30,27 @@ namespace odsgd {
 #define ODSGD_BATCH 8  // gradient loads in flight per thread and vector
 #endif
 #ifndef ODSGD_UNROLL
-#define ODSGD_UNROLL 1  // vectors per thread per tile
+#define ODSGD_UNROLL 2  // vectors per thread per tile
+#endif
+#ifndef ODSGD_GRAD_LOAD
+#define ODSGD_GRAD_LOAD 1  // 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching
+#endif
+#ifndef ODSGD_STORE
+#define ODSGD_STORE 0  // 0 streaming (st.global.cs), 1 default caching
+#endif
+#ifndef ODSGD_MIN_CTAS
+#define ODSGD_MIN_CTAS 0  // > 0: __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS) on the server kernel
+#endif
+#ifndef ODSGD_MAX_BLOCK
+#define ODSGD_MAX_BLOCK 256
 #endif
 constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
+#if ODSGD_MIN_CTAS > 0
+#define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
+#else
+#define ODSGD_SERVER_BOUNDS
+#endif
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
 
@@ -94,15 +115,49 @@ __device__ __forceinline__ Vec<1> load_stream<1>(const float* p) {
     return Vec<1>{{__ldcs(p)}};
 }
 
+// Gradients (and the backup weights of the local kernel) are never written by the kernel
+// that reads them, so they may also go through the read-only path.
+template <int NL>
+__device__ __forceinline__ Vec<NL> load_grad(const float* p);
+template <>
+__device__ __forceinline__ Vec<4> load_grad<4>(const float* p) {
+#if ODSGD_GRAD_LOAD == 1
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+#elif ODSGD_GRAD_LOAD == 2
+    const float4 t = *reinterpret_cast<const float4*>(p);
+#else
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
+#endif
+    return Vec<4>{{t.x, t.y, t.z, t.w}};
+}
+template <>
+__device__ __forceinline__ Vec<1> load_grad<1>(const float* p) {
+#if ODSGD_GRAD_LOAD == 1
+    return Vec<1>{{__ldg(p)}};
+#elif ODSGD_GRAD_LOAD == 2
+    return Vec<1>{{*p}};
+#else
+    return Vec<1>{{__ldcs(p)}};
+#endif
+}
+
 template <int NL>
 __device__ __forceinline__ void store_stream(float* p, const Vec<NL>& a);
 template <>
 __device__ __forceinline__ void store_stream<4>(float* p, const Vec<4>& a) {
+#if ODSGD_STORE == 1
+    *reinterpret_cast<float4*>(p) = make_float4(a.e[0], a.e[1], a.e[2], a.e[3]);
+#else
     __stcs(reinterpret_cast<float4*>(p), make_float4(a.e[0], a.e[1], a.e[2], a.e[3]));
+#endif
 }
 template <>
 __device__ __forceinline__ void store_stream<1>(float* p, const Vec<1>& a) {
+#if ODSGD_STORE == 1
+    *p = a.e[0];
+#else
     __stcs(p, a.e[0]);
+#endif
 }
 
 // ------------------------------------------------------------------ arithmetic
@@ -173,7 +228,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                 const float* gp = a.g[m0 + j];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    if (ok[u]) t[j][u] = load_stream<NL>(gp + off[u]);
+                    if (ok[u]) t[j][u] = load_grad<NL>(gp + off[u]);
                 }
             }
         }
@@ -241,7 +296,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 }
 
 template <bool DET, int NL, int LOCAL, int RULE>
-__global__ void server_kernel(const __grid_constant__ ServerArgs a) {
+__global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * kUnroll;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
@@ -270,8 +325,8 @@ __global__ void server_kernel(const __grid_constant__ ServerArgs a) {
 // ------------------------------------------------------------------ local kernel
 template <bool DET, int NL, int RULE>
 __device__ __forceinline__ void local_vector(const LocalArgs& a, unsigned long long off) {
-    const Vec<NL> w = load_stream<NL>(a.w_bak + off);
-    const Vec<NL> g = load_stream<NL>(a.g + off);
+    const Vec<NL> w = load_grad<NL>(a.w_bak + off);
+    const Vec<NL> g = load_grad<NL>(a.g + off);
     Vec<NL> xv, msv, xo;
     if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(a.x + off);
     if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms + off);
@@ -297,7 +352,7 @@ __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
 // ------------------------------------------------------------------ ASGD kernel
 template <bool DET, int NL>
 __device__ __forceinline__ void asgd_vector(const AsgdArgs& a, unsigned long long off) {
-    const Vec<NL> g = load_stream<NL>(a.g + off);
+    const Vec<NL> g = load_grad<NL>(a.g + off);
     const Vec<NL> w = load_stream<NL>(a.w + off);
     const Vec<NL> v = load_stream<NL>(a.v + off);
     Vec<NL> wn, vn;
