@@ -41,6 +41,29 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_traffic(step_bytes):
+    """DRAM bytes per launch from the committed ncu capture of the fused kernel, scaled by the
+    algorithmic bytes (traffic grows in proportion: every stream is touched once).  None when the
+    kernel source has changed since the counters were taken."""
+    import hashlib
+    import re
+
+    try:
+        note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_alexnet_m8.md")).read()
+        src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
+        ratio = float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1))
+        sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1)
+    except (OSError, AttributeError, ValueError):
+        return None
+    if hashlib.sha256(src).hexdigest() != sha:
+        return None
+    return ratio * step_bytes
+
+
+def workload_label(wl, n_workers):
+    return f"{wl.name}-shaped parameter set, M={n_workers} workers, fused global+local update"
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -122,8 +145,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": info["value"], "unit": "GB/s", "n_gpus": args.gpus,
         "steps": done, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{wl.name} M={n_workers} (CPU oracle on a bounded sample)", "n_params": wl.n_params,
-                   "n_workers": n_workers, "sample_elems": min(args.cpu_sample, wl.arena_len)},
+        "config": {"workload": workload_label(wl, n_workers), "n_params": wl.n_params, "n_tensors": wl.n_tensors,
+                   "n_workers": n_workers, "sample_elems": min(args.cpu_sample, wl.arena_len),
+                   "note": "CPU oracle, single thread, on a bounded sample of the workload"},
         "cpu_baseline": {k: info[k] for k in ("value", "unit", "cores", "kind", "sample")},
         "e2e": {"value": info["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "params_per_s": info["params_per_s"], "host": info["host"],
@@ -267,7 +291,7 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{wl.name}-shaped parameter set, M={M} workers, fused global+local update",
+        "config": {"workload": workload_label(wl, M),
                    "n_params": P, "n_tensors": wl.n_tensors, "n_workers": M,
                    "bytes_per_step": step_bytes, "l2": l2_note,
                    "flavour": "deterministic" if args.deterministic else "default (FMA contraction allowed)",
@@ -276,7 +300,7 @@ def run_cuda(args):
                    "power_w_max": ck.get("power_w_max"), "samples": ck.get("samples"), "source": ck.get("source")},
         "e2e": e2e, "gpu_launches": gpu_launches,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": f"of {peak_src}", "kernel": "server_kernel (fused, one local)",
+                     "traffic": measured_traffic(step_bytes), "peak_source": f"of {peak_src}", "kernel": "server_kernel (fused, one local)",
                      "kernel_ms": kernel_ms, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
         "cpu_baseline": cpu,
         "params_per_s": P * args.steps * world / (agg["ms"] * 1e-3),
