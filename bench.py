@@ -75,6 +75,8 @@ def parse_args():
     ap.add_argument("--deterministic", action="store_true", help="time the one-rounding-per-operator flavour")
     ap.add_argument("--block", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--graph", type=int, default=0,
+                    help="capture this many steps (even) in one CUDA graph and replay it; for the small, launch-bound sets")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra-kernels", action="store_true")
@@ -204,21 +206,44 @@ def run_cuda(args):
     for _ in range(max(3, args.warmup)):
         ctx.fused_update(grads, 0, stream)
     torch.cuda.synchronize()
-    barrier(dev)
-    torch.cuda.synchronize()
-    launches_before = ctx.launch_count
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    with ClockSampler(dev.index or 0) as clocks:
-        ev[0].record(stream)
-        for k in range(args.steps):
-            ctx.fused_update(grads, 0, stream)
-            ev[k + 1].record(stream)
+    graph = None
+    if args.graph:
+        if args.graph % 2 or args.steps % args.graph:
+            raise SystemExit("--graph must be even (the weight halves swap every step) and divide --steps")
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(args.graph):
+                ctx.fused_update(grads, 0)  # lands on the capturing stream
+        for _ in range(3):
+            graph.replay()
         torch.cuda.synchronize()
     barrier(dev)
     torch.cuda.synchronize()
-    gpu_launches = ctx.launch_count - launches_before
+    launches_before = ctx.launch_count
+    if graph is None:
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        with ClockSampler(dev.index or 0) as clocks:
+            ev[0].record(stream)
+            for k in range(args.steps):
+                ctx.fused_update(grads, 0, stream)
+                ev[k + 1].record(stream)
+            torch.cuda.synchronize()
+        gpu_launches = ctx.launch_count - launches_before
+        per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    else:
+        replays = args.steps // args.graph
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
+        with ClockSampler(dev.index or 0) as clocks:
+            ev[0].record(stream)
+            for k in range(replays):
+                graph.replay()
+                ev[k + 1].record(stream)
+            torch.cuda.synchronize()
+        gpu_launches = args.steps  # one kernel node per captured step, replayed
+        per_step = [ev[k].elapsed_time(ev[k + 1]) / args.graph for k in range(replays)]
+    barrier(dev)
+    torch.cuda.synchronize()
     total_ms = ev[0].elapsed_time(ev[-1])
-    per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
     agg = aggregate(total_ms, float(step_bytes) * args.steps, dev if world > 1 else None)
     ms_per_step = agg["ms"] / args.steps
     value = agg["units"] / (agg["ms"] * 1e-3) / 1e9
@@ -295,6 +320,7 @@ def run_cuda(args):
                    "n_params": P, "n_tensors": wl.n_tensors, "n_workers": M,
                    "bytes_per_step": step_bytes, "l2": l2_note,
                    "flavour": "deterministic" if args.deterministic else "default (FMA contraction allowed)",
+                   "launch": f"CUDA graph of {args.graph} steps, replayed" if args.graph else "one launch per step from the host",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),
                    "power_w_max": ck.get("power_w_max"), "samples": ck.get("samples"), "source": ck.get("source")},

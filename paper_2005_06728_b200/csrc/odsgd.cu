@@ -45,8 +45,9 @@ namespace {
 
 thread_local std::string g_create_err;
 
-constexpr int kDefaultBlock = 256;
-// Grid cap of the server kernel in CTAs per SM.  More CTAs than can be resident (two at this
+constexpr int kDefaultBlock = 256;       // server kernel
+constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels (measured best with 4 vectors per thread)
+// Grid cap of the kernels in CTAs per SM.  More CTAs than can be resident (two at this
 // register count) measured 1-2 % faster than an exactly persistent grid: late SMs pick up
 // the remaining tiles.
 constexpr int kServerCtasPerSm = 64;
@@ -191,7 +192,7 @@ int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, 
 
 template <bool DET, int NL, int RULE>
 int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = local_kernel<DET, NL, RULE>;
     static int cached_block = 0, cached_res = 0;
     if (cached_block != block) {
@@ -199,7 +200,7 @@ int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
         cached_block = block;
     }
     if (cached_res == 0) return too_wide(c, block);
-    kernel<<<grid_for(c, a.n, NL, block, 1, cached_res), block, 0, st>>>(a);
+    kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
     return after_launch(c, "local kernel launch");
 }
 
@@ -220,7 +221,7 @@ int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, cudaStream_t st) {
 
 template <bool DET, int NL>
 int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = asgd_kernel<DET, NL>;
     static int cached_block = 0, cached_res = 0;
     if (cached_block != block) {
@@ -228,7 +229,7 @@ int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
         cached_block = block;
     }
     if (cached_res == 0) return too_wide(c, block);
-    kernel<<<grid_for(c, a.n, NL, block, 1, cached_res), block, 0, st>>>(a);
+    kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
     return after_launch(c, "asgd kernel launch");
 }
 

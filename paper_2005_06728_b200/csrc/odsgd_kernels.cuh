@@ -44,8 +44,12 @@ namespace odsgd {
 #ifndef ODSGD_MAX_BLOCK
 #define ODSGD_MAX_BLOCK 256
 #endif
+#ifndef ODSGD_SMALL_UNROLL
+#define ODSGD_SMALL_UNROLL 4  // vectors per thread per tile in the local and ASGD kernels
+#endif
 constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
+constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
 #if ODSGD_MIN_CTAS > 0
 #define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
 #else
@@ -323,55 +327,106 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
 }
 
 // ------------------------------------------------------------------ local kernel
-template <bool DET, int NL, int RULE>
-__device__ __forceinline__ void local_vector(const LocalArgs& a, unsigned long long off) {
-    const Vec<NL> w = load_grad<NL>(a.w_bak + off);
-    const Vec<NL> g = load_grad<NL>(a.g + off);
-    Vec<NL> xv, msv, xo;
-    if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(a.x + off);
-    if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms + off);
+// Few streams per element (2-4 reads, 1-2 writes): each thread takes kSmallUnroll vectors per
+// tile and issues all their loads before the first store, which is what a plain copy needs
+// to approach the copy ceiling of the part.
+template <bool DET, int NL, int RULE, int U>
+__device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned long long (&off)[U],
+                                              const bool (&ok)[U]) {
+    Vec<NL> w[U], g[U], xv[U], msv[U];
 #pragma unroll
-    for (int l = 0; l < NL; ++l) xo.e[l] = local_rule<DET, RULE>(w.e[l], g.e[l], xv.e[l], msv.e[l], a.lp);
-    store_stream<NL>(a.x + off, xo);
-    if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms + off, msv);
+    for (int u = 0; u < U; ++u) {
+        if (ok[u]) {
+            w[u] = load_grad<NL>(a.w_bak + off[u]);
+            g[u] = load_grad<NL>(a.g + off[u]);
+            if (RULE != ODSGD_LOCAL_SGD) xv[u] = load_stream<NL>(a.x + off[u]);
+            if (RULE == ODSGD_LOCAL_DC_A) msv[u] = load_stream<NL>(a.ms + off[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        Vec<NL> xo;
+#pragma unroll
+        for (int l = 0; l < NL; ++l) xo.e[l] = local_rule<DET, RULE>(w[u].e[l], g[u].e[l], xv[u].e[l], msv[u].e[l], a.lp);
+        store_stream<NL>(a.x + off[u], xo);
+        if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms + off[u], msv[u]);
+    }
 }
 
 template <bool DET, int NL, int RULE>
 __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
     const unsigned long long nvec = a.n / NL;
-    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        local_vector<DET, NL, RULE>(a, i * NL);
+    const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
+    const unsigned long long stride = (unsigned long long)gridDim.x * tile;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * tile; base < nvec; base += stride) {
+        unsigned long long off[kSmallUnroll];
+        bool ok[kSmallUnroll];
+#pragma unroll
+        for (int u = 0; u < kSmallUnroll; ++u) {
+            const unsigned long long i = base + (unsigned long long)u * blockDim.x + threadIdx.x;
+            ok[u] = i < nvec;
+            off[u] = i * NL;
+        }
+        local_vectors<DET, NL, RULE, kSmallUnroll>(a, off, ok);
     }
     if (NL > 1) {
         const unsigned long long done = nvec * NL;
-        if (blockIdx.x == 0 && done + threadIdx.x < a.n) local_vector<DET, 1, RULE>(a, done + threadIdx.x);
+        if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
+            const unsigned long long off1[1] = {done + threadIdx.x};
+            const bool ok1[1] = {true};
+            local_vectors<DET, 1, RULE, 1>(a, off1, ok1);
+        }
     }
 }
 
 // ------------------------------------------------------------------ ASGD kernel
-template <bool DET, int NL>
-__device__ __forceinline__ void asgd_vector(const AsgdArgs& a, unsigned long long off) {
-    const Vec<NL> g = load_grad<NL>(a.g + off);
-    const Vec<NL> w = load_stream<NL>(a.w + off);
-    const Vec<NL> v = load_stream<NL>(a.v + off);
-    Vec<NL> wn, vn;
+template <bool DET, int NL, int U>
+__device__ __forceinline__ void asgd_vectors(const AsgdArgs& a, const unsigned long long (&off)[U], const bool (&ok)[U]) {
+    Vec<NL> g[U], w[U], v[U];
 #pragma unroll
-    for (int l = 0; l < NL; ++l) server_rule<DET>(g.e[l], w.e[l], v.e[l], a.lr, a.momentum, a.wd, wn.e[l], vn.e[l]);
-    store_stream<NL>(a.v + off, vn);
-    store_stream<NL>(a.w + off, wn);
+    for (int u = 0; u < U; ++u) {
+        if (ok[u]) {
+            g[u] = load_grad<NL>(a.g + off[u]);
+            w[u] = load_stream<NL>(a.w + off[u]);
+            v[u] = load_stream<NL>(a.v + off[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        if (!ok[u]) continue;
+        Vec<NL> wn, vn;
+#pragma unroll
+        for (int l = 0; l < NL; ++l)
+            server_rule<DET>(g[u].e[l], w[u].e[l], v[u].e[l], a.lr, a.momentum, a.wd, wn.e[l], vn.e[l]);
+        store_stream<NL>(a.v + off[u], vn);
+        store_stream<NL>(a.w + off[u], wn);
+    }
 }
 
 template <bool DET, int NL>
 __global__ void asgd_kernel(const __grid_constant__ AsgdArgs a) {
     const unsigned long long nvec = a.n / NL;
-    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += stride) {
-        asgd_vector<DET, NL>(a, i * NL);
+    const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
+    const unsigned long long stride = (unsigned long long)gridDim.x * tile;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * tile; base < nvec; base += stride) {
+        unsigned long long off[kSmallUnroll];
+        bool ok[kSmallUnroll];
+#pragma unroll
+        for (int u = 0; u < kSmallUnroll; ++u) {
+            const unsigned long long i = base + (unsigned long long)u * blockDim.x + threadIdx.x;
+            ok[u] = i < nvec;
+            off[u] = i * NL;
+        }
+        asgd_vectors<DET, NL, kSmallUnroll>(a, off, ok);
     }
     if (NL > 1) {
         const unsigned long long done = nvec * NL;
-        if (blockIdx.x == 0 && done + threadIdx.x < a.n) asgd_vector<DET, 1>(a, done + threadIdx.x);
+        if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
+            const unsigned long long off1[1] = {done + threadIdx.x};
+            const bool ok1[1] = {true};
+            asgd_vectors<DET, 1, 1>(a, off1, ok1);
+        }
     }
 }
 

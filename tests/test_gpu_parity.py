@@ -299,6 +299,28 @@ def test_host_buffer_entry_point(cuda_device):
         assert torch.equal(out, lr_[1].cpu()) and torch.equal(local[1], lr_[1])
 
 
+def test_cuda_graph_replay_matches_eager_calls(cuda_device):
+    """An even number of steps captured in a CUDA graph (the weight halves swap every step)
+    replays to the same bits as the same steps issued one by one."""
+    wl = W.workload("lenet5")
+    a, _, va, la = _ctx_for(wl, True, True)
+    b, _, vb, lb = _ctx_for(wl, True, True)
+    grads = W.make_grads(wl, 0, DEV)
+    a.fused_update(grads, 0), a.fused_update(grads, 0)  # warm-up outside the capture
+    b.fused_update(grads, 0), b.fused_update(grads, 0)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(4):
+            a.fused_update(grads, 0)
+    for _ in range(4):  # the capture itself runs nothing: 16 steps happen here
+        graph.replay()
+    for _ in range(16):
+        b.fused_update(grads, 0)
+    torch.cuda.synchronize()
+    assert torch.equal(a.weights(), b.weights()) and torch.equal(va, vb) and torch.equal(la[0], lb[0])
+
+
 # ------------------------------------------------------------------ whole configurations
 
 def _trajectory(wl, det, iterations, check_every=1):
