@@ -48,6 +48,10 @@ def lib() -> ctypes.CDLL:
             "oracle_asgd_step": [f32p, sz, f32p, f32p, cf, cf, cf],
             "oracle_local_update_dc_c": [f32p, f32p, f32p, sz, f32p, cf, cf],
             "oracle_local_update_dc_a": [f32p, f32p, f32p, f32p, sz, f32p, cf, cf, cf, cf],
+            "oracle_global_update_mult": [pp32, ci, sz, f32p, f32p, f32p, cf, cf, cf,
+                                          ctypes.POINTER(sz), sz, f32p, f32p],
+            "oracle_dcasgd_step_c": [f32p, sz, f32p, f32p, cf, cf],
+            "oracle_dcasgd_step_a": [f32p, sz, f32p, f32p, f32p, cf, cf, cf, cf],
             "oracle_global_update_f64": [pp64, ci, sz, f64p, f64p, f64p, cd, cd, cd],
             "oracle_local_update_f64": [f64p, f64p, sz, f64p, cd],
             "oracle_asgd_step_f64": [f64p, sz, f64p, f64p, cd, cd, cd],
@@ -158,6 +162,49 @@ def local_update_dc_a(w_bak: np.ndarray, g: np.ndarray, x_prev: np.ndarray,
                                    _ptr(mean_square, ctypes.c_float), n,
                                    _ptr(x, ctypes.c_float), local_lr, lam, m, eps)
     return x
+
+
+def global_update_mult(grads: Sequence[np.ndarray], w: np.ndarray, v: np.ndarray, *, lr: float,
+                       momentum: float, wd: float, offsets: Sequence[int], lr_mult: np.ndarray,
+                       wd_mult: np.ndarray, w_prev: Optional[np.ndarray] = None) -> None:
+    """Algorithm 1's update with per-tensor learning-rate and weight-decay multipliers, in place."""
+    n = _chk(w, np.float32, "w").shape[0]
+    _chk(v, np.float32, "v", n)
+    for m, g in enumerate(grads):
+        _chk(g, np.float32, f"grads[{m}]", n)
+    nt = len(offsets) - 1
+    _chk(lr_mult, np.float32, "lr_mult", nt)
+    _chk(wd_mult, np.float32, "wd_mult", nt)
+    if w_prev is not None:
+        _chk(w_prev, np.float32, "w_prev", n)
+    offs = (ctypes.c_size_t * len(offsets))(*[int(o) for o in offsets])
+    rc = lib().oracle_global_update_mult(_ptr_table(grads, ctypes.c_float), len(grads), n,
+                                         _ptr(w, ctypes.c_float), _ptr(v, ctypes.c_float),
+                                         _ptr(w_prev, ctypes.c_float), lr, momentum, wd, offs, nt,
+                                         _ptr(lr_mult, ctypes.c_float), _ptr(wd_mult, ctypes.c_float))
+    if rc != 0:
+        raise ValueError("oracle_global_update_mult: bad worker count or offsets")
+
+
+def dcasgd_step_c(g: np.ndarray, w: np.ndarray, w_bak_m: np.ndarray, *, lr: float, lam: float) -> None:
+    """Eq. 4 applied at the server to one arriving gradient; w and the worker's backup in place."""
+    n = _chk(w, np.float32, "w").shape[0]
+    _chk(g, np.float32, "g", n)
+    _chk(w_bak_m, np.float32, "w_bak_m", n)
+    lib().oracle_dcasgd_step_c(_ptr(g, ctypes.c_float), n, _ptr(w, ctypes.c_float),
+                               _ptr(w_bak_m, ctypes.c_float), lr, lam)
+
+
+def dcasgd_step_a(g: np.ndarray, w: np.ndarray, w_bak_m: np.ndarray, mean_square: np.ndarray, *,
+                  lr: float, lam: float, m: float, eps: float) -> None:
+    """Eq. 6 then Eq. 5 applied at the server to one arriving gradient, in place."""
+    n = _chk(w, np.float32, "w").shape[0]
+    _chk(g, np.float32, "g", n)
+    _chk(w_bak_m, np.float32, "w_bak_m", n)
+    _chk(mean_square, np.float32, "mean_square", n)
+    lib().oracle_dcasgd_step_a(_ptr(g, ctypes.c_float), n, _ptr(w, ctypes.c_float),
+                               _ptr(w_bak_m, ctypes.c_float), _ptr(mean_square, ctypes.c_float),
+                               lr, lam, m, eps)
 
 
 def global_update_f64(grads: Sequence[np.ndarray], w: np.ndarray, v: np.ndarray, *, lr: float,

@@ -157,6 +157,88 @@ int oracle_local_update_dc_a(const float* w_bak, const float* g, const float* x_
     return 0;
 }
 
+// ---------------------------------------------------------------- per-tensor multipliers
+// The stock updater of the framework the paper used scales the learning rate and the
+// weight decay per parameter tensor (lr_mult, wd_mult; biases and batch-norm scales
+// commonly get wd_mult = 0).  Tensor t owns elements [offsets[t], offsets[t+1]).
+//   lr_t = lr * lr_mult[t];  wd_t = wd * wd_mult[t];  then Algorithm 1's update with lr_t, wd_t.
+int oracle_global_update_mult(const float* const* grads, int n_workers, size_t n,
+                              float* w, float* v, float* w_prev,
+                              float lr, float momentum, float wd,
+                              const size_t* offsets, size_t n_tensors,
+                              const float* lr_mult, const float* wd_mult)
+{
+    if (n_workers < 1 || n_tensors < 1 || offsets[0] != 0 || offsets[n_tensors] != n) return -1;
+    const float inv_m = 1.0f / (float)n_workers;
+    for (size_t t = 0; t < n_tensors; ++t) {
+        const float lr_t = lr * lr_mult[t];
+        const float wd_t = wd * wd_mult[t];
+        for (size_t i = offsets[t]; i < offsets[t + 1]; ++i) {
+            float s = grads[0][i];
+            for (int m = 1; m < n_workers; ++m) s = s + grads[m][i];
+            const float gbar = s * inv_m;
+            const float decay = wd_t * w[i];
+            const float d = gbar + decay;
+            const float keep = momentum * v[i];
+            const float step = lr_t * d;
+            const float v_new = keep - step;
+            const float w_new = w[i] + v_new;
+            if (w_prev) w_prev[i] = w[i];
+            v[i] = v_new;
+            w[i] = w_new;
+        }
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------- DC-ASGD at the server
+// The paper's fourth comparison algorithm (Section 4.1): Eq. 4 / Eq. 5 applied by the
+// parameter server to each arriving gradient.  w is the current global vector (the
+// paper's w_{t+tau}); w_bak_m is the copy worker m pulled before computing g (the
+// paper's w_t).  After the step worker m pulls again, so its backup becomes the new w.
+// No momentum and no weight decay appear in Eq. 4 / Eq. 5 (Section 4.1 sets momentum 0).
+//   w <- w - eta * (g + lambda * g*g * (w - w_bak_m));   w_bak_m <- w
+int oracle_dcasgd_step_c(const float* g, size_t n, float* w, float* w_bak_m, float lr, float lambda)
+{
+    for (size_t i = 0; i < n; ++i) {
+        const float diff = w[i] - w_bak_m[i];
+        const float gg = g[i] * g[i];
+        const float lgg = lambda * gg;
+        const float comp = lgg * diff;
+        const float d = g[i] + comp;
+        const float step = lr * d;
+        const float w_new = w[i] - step;
+        w[i] = w_new;
+        w_bak_m[i] = w_new;
+    }
+    return 0;
+}
+
+// Eq. 6 then Eq. 5 at the server; mean_square is the server's single running average.
+int oracle_dcasgd_step_a(const float* g, size_t n, float* w, float* w_bak_m, float* mean_square,
+                         float lr, float lambda, float m, float eps)
+{
+    const float one_minus_m = 1.0f - m;
+    for (size_t i = 0; i < n; ++i) {
+        const float gg = g[i] * g[i];
+        const float a = m * mean_square[i];
+        const float b = one_minus_m * gg;
+        const float ms = a + b;
+        mean_square[i] = ms;
+        const float den = std::sqrt(ms + eps);
+        const float lam = lambda / den;
+        const float diff = w[i] - w_bak_m[i];
+        const float lgg = lam * gg;
+        const float comp = lgg * diff;
+        const float d = g[i] + comp;
+        const float step = lr * d;
+        const float w_new = w[i] - step;
+        w[i] = w_new;
+        w_bak_m[i] = w_new;
+    }
+    return 0;
+}
+
 // ---------------------------------------------------------------- fp64 twins
 // Same rules, all arithmetic in binary64 on binary64 state.  Used only to
 // bound the rounding error of the fp32 rules in the tests.

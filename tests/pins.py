@@ -48,6 +48,19 @@ class Impl:
         """returns (x, ms_new)"""
         raise NotImplementedError
 
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult
+                           ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """returns (w_new, v_new, w_prev)"""
+        raise NotImplementedError
+
+    def dcasgd_step_c(self, g, w, bak, lr, lam) -> Tuple[np.ndarray, np.ndarray]:
+        """returns (w_new, bak_new)"""
+        raise NotImplementedError
+
+    def dcasgd_step_a(self, g, w, bak, ms, lr, lam, m, eps) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """returns (w_new, bak_new, ms_new)"""
+        raise NotImplementedError
+
 
 def a32(x) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(x, dtype=np.float32).reshape(-1))
@@ -416,7 +429,92 @@ def pin_dc_reductions(impl: Impl, seed: int = 55) -> None:
     np.testing.assert_allclose(xc, e, rtol=0, atol=1e-6)
 
 
+# ----------------------------------------------------------------- per-tensor multipliers
+
+def pin_multipliers(impl: Impl, seed: int = 66) -> None:
+    """impl.global_update_mult(grads, w, v, lr, mu, wd, offsets, lr_mult, wd_mult) -> (w, v, w_prev)"""
+    g = read_golden("per_tensor_multipliers.txt")
+    offs = [int(o) for o in g["offsets"]]
+    w1, v1, wp = impl.global_update_mult([a32(g["g0"]), a32(g["g1"])], a32(g["w"]), a32(g["v"]),
+                                         float(g["lr"][0]), float(g["momentum"][0]), float(g["wd"][0]),
+                                         offs, a32(g["lr_mult"]), a32(g["wd_mult"]))
+    assert np.array_equal(w1, a32(g["w1"])), ("hand example, w", w1)
+    assert np.array_equal(v1, a32(g["v1"])), ("hand example, v", v1)
+    assert np.array_equal(wp, a32(g["w"]))
+    # all multipliers 1: the plain rule, bit for bit; in general: tensor by tensor the plain
+    # rule with that tensor's scaled hyper-parameters
+    rng = np.random.default_rng(seed)
+    sizes = [5, 64, 1, 300, 7, 2048]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).tolist()
+    n = offs[-1]
+    w, v = a32(rng.normal(0, 1, n)), a32(rng.normal(0, 0.1, n))
+    grads = [a32(rng.normal(0, 0.3, n)) for _ in range(3)]
+    lr, mu, wd = 0.07, 0.9, 2e-3
+    ones = np.ones(len(sizes), F32)
+    wa, va, _ = impl.global_update_mult(grads, w.copy(), v.copy(), lr, mu, wd, offs, ones, ones)
+    wb, vb, _ = impl.global_update(grads, w.copy(), v.copy(), lr, mu, wd)
+    assert_same_bits(wa, wb, "multipliers all 1 (w)")
+    assert_same_bits(va, vb, "multipliers all 1 (v)")
+    lm = a32([1.0, 0.5, 2.0, 0.1, 0.0, 1.5])
+    wm = a32([1.0, 0.0, 0.0, 3.0, 1.0, 0.25])
+    wa, va, _ = impl.global_update_mult(grads, w.copy(), v.copy(), lr, mu, wd, offs, lm, wm)
+    for t, (a, b) in enumerate(zip(offs[:-1], offs[1:])):
+        lr_t = float(F32(lr) * lm[t])
+        wd_t = float(F32(wd) * wm[t])
+        ws, vs, _ = impl.global_update([x[a:b].copy() for x in grads], w[a:b].copy(), v[a:b].copy(), lr_t, mu, wd_t)
+        assert_same_bits(wa[a:b], ws, f"tensor {t} against the plain rule (w)")
+        assert_same_bits(va[a:b], vs, f"tensor {t} against the plain rule (v)")
+    a, b = offs[4], offs[5]  # lr_mult = 0: only momentum moves the weights
+    np.testing.assert_array_equal(va[a:b], F32(mu) * v[a:b])
+
+
+# ----------------------------------------------------------------- DC-ASGD at the server
+
+def pin_dcasgd_server(impl: Impl, seed: int = 77) -> None:
+    """impl.dcasgd_step_c(g, w, bak, lr, lam) -> (w, bak);
+    impl.dcasgd_step_a(g, w, bak, ms, lr, lam, m, eps) -> (w, bak, ms)"""
+    g = read_golden("dc_local_update.txt")
+    # same arithmetic as the worker-side rule with (w, backup) in the roles (w_bak, x_prev)
+    w1, bak1 = impl.dcasgd_step_c(a32(g["c_g"]), a32(g["c_w_bak"]), a32(g["c_x_prev"]),
+                                  float(g["c_eta"][0]), float(g["c_lambda"][0]))
+    assert np.array_equal(w1, a32(g["c_x"])), ("Eq. 4 at the server", w1)
+    assert np.array_equal(bak1, w1), "the worker pulls the new weights after its gradient is applied"
+    w1, bak1, ms1 = impl.dcasgd_step_a(a32(g["a_g"]), a32(g["a_w_bak"]), a32(g["a_x_prev"]), a32(g["a_ms"]),
+                                       float(g["a_eta"][0]), float(g["a_lambda"][0]), float(g["a_m"][0]),
+                                       float(g["a_eps"][0]))
+    assert np.array_equal(w1, a32(g["a_x"])) and np.array_equal(ms1, a32(g["a_ms_new"]))
+    assert np.array_equal(bak1, w1)
+    rng = np.random.default_rng(seed)
+    n = 500
+    w = a32(rng.normal(0, 1, n))
+    bak = a32(w + rng.normal(0, 0.05, n))
+    gr = a32(rng.normal(0, 0.5, n))
+    # lambda = 0, or a worker that is not behind: plain SGD, i.e. the ASGD step without momentum and decay
+    plain, _ = impl.asgd_step(gr, w.copy(), np.zeros(n, F32), 0.1, 0.0, 0.0)
+    w1, _ = impl.dcasgd_step_c(gr, w.copy(), bak.copy(), 0.1, 0.0)
+    assert_same_bits(w1, plain, "lambda = 0")
+    w1, b1 = impl.dcasgd_step_c(gr, w.copy(), w.copy(), 0.1, 2.0)
+    assert_same_bits(w1, plain, "no delay")
+    # bit-identical to the (separately pinned) worker-side rule
+    w1, b1 = impl.dcasgd_step_c(gr, w.copy(), bak.copy(), 0.1, 2.0)
+    assert_same_bits(w1, impl.local_update_dc_c(w, gr, bak, 0.1, 2.0), "server rule vs worker rule, Eq. 4")
+    ms = a32(rng.uniform(0.01, 1, n))
+    w1, b1, ms1 = impl.dcasgd_step_a(gr, w.copy(), bak.copy(), ms.copy(), 0.1, 2.0, 0.95, 1e-7)
+    xe, mse = impl.local_update_dc_a(w, gr, bak, ms.copy(), 0.1, 2.0, 0.95, 1e-7)
+    assert_same_bits(w1, xe, "server rule vs worker rule, Eq. 5")
+    assert_same_bits(ms1, mse, "Eq. 6 state")
+    assert_same_bits(b1, w1, "backup after the step")
+    # two workers taking turns: the one that pulled last is not behind
+    wa, ba = impl.dcasgd_step_c(gr, w.copy(), w.copy(), 0.1, 2.0)       # worker 0, fresh
+    g2 = a32(rng.normal(0, 0.5, n))
+    wb, bb = impl.dcasgd_step_c(g2, wa.copy(), w.copy(), 0.1, 2.0)      # worker 1 still holds w
+    diff = wa.astype(np.float64) - w
+    expect = wa - 0.1 * (g2 + 2.0 * g2.astype(np.float64) ** 2 * diff)
+    np.testing.assert_allclose(wb, expect, rtol=0, atol=1e-6)
+
+
 CORE_PINS = (pin_worked_example, pin_rounding_order, pin_ssgd_quadratic_closed_form,
              pin_odsgd_quadratic_matrix_form, pin_odsgd_special_cases, pin_invariants,
              pin_special_values, pin_exact_rational)
 DC_PINS = (pin_dc_worked_example, pin_dc_reductions)
+EXT_PINS = (pin_multipliers, pin_dcasgd_server)

@@ -43,6 +43,24 @@ class OracleImpl(Impl):
         return x, ms
 
 
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        w, v = w.copy(), v.copy()
+        wp = np.empty_like(w)
+        oracle.global_update_mult(list(grads), w, v, lr=lr, momentum=momentum, wd=wd, offsets=offsets,
+                                  lr_mult=lr_mult, wd_mult=wd_mult, w_prev=wp)
+        return w, v, wp
+
+    def dcasgd_step_c(self, g, w, bak, lr, lam):
+        w, bak = w.copy(), bak.copy()
+        oracle.dcasgd_step_c(g, w, bak, lr=lr, lam=lam)
+        return w, bak
+
+    def dcasgd_step_a(self, g, w, bak, ms, lr, lam, m, eps):
+        w, bak, ms = w.copy(), bak.copy(), ms.copy()
+        oracle.dcasgd_step_a(g, w, bak, ms, lr=lr, lam=lam, m=m, eps=eps)
+        return w, bak, ms
+
+
 class NumpyImpl(Impl):
     """The rules restated with numpy fp32 array ops; the base the wrong variants are cut from."""
 
@@ -81,10 +99,29 @@ class NumpyImpl(Impl):
         return w_bak - F32(local_lr) * (g + (lam_t * (g * g)) * (w_bak - x_prev)), ms
 
 
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        gbar = self._sum(grads) * (F32(1.0) / F32(len(grads)))
+        lr_e, wd_e = np.empty_like(w), np.empty_like(w)
+        for t, (a, b) in enumerate(zip(offsets[:-1], offsets[1:])):
+            lr_e[a:b] = F32(lr) * lr_mult[t]
+            wd_e[a:b] = F32(wd) * wd_mult[t]
+        d = gbar + wd_e * w
+        vn = F32(momentum) * v - lr_e * d
+        return w + vn, vn, w.copy()
+
+    def dcasgd_step_c(self, g, w, bak, lr, lam):
+        wn = self.local_update_dc_c(w, g, bak, lr, lam)
+        return wn, wn.copy()
+
+    def dcasgd_step_a(self, g, w, bak, ms, lr, lam, m, eps):
+        wn, msn = self.local_update_dc_a(w, g, bak, ms, lr, lam, m, eps)
+        return wn, wn.copy(), msn
+
+
 ORACLE = OracleImpl()
 
 
-@pytest.mark.parametrize("pin", pins.CORE_PINS + pins.DC_PINS, ids=lambda f: f.__name__)
+@pytest.mark.parametrize("pin", pins.CORE_PINS + pins.DC_PINS + pins.EXT_PINS, ids=lambda f: f.__name__)
 def test_oracle_pin(pin):
     pin(ORACLE)
 
@@ -110,7 +147,7 @@ def test_fp64_asgd_twin_matches_one_worker_server_step():
     np.testing.assert_allclose(v1, v2, rtol=1e-15)
 
 
-@pytest.mark.parametrize("pin", pins.CORE_PINS + pins.DC_PINS, ids=lambda f: f.__name__)
+@pytest.mark.parametrize("pin", pins.CORE_PINS + pins.DC_PINS + pins.EXT_PINS, ids=lambda f: f.__name__)
 def test_numpy_restatement_passes_too(pin):
     pin(NumpyImpl())
 
@@ -325,6 +362,46 @@ class DcEpsOutsideRoot(NumpyImpl):
                          ids=lambda c: c.__name__)
 def test_planted_dc_mistake_is_caught(mutant):
     assert _rejected_by(mutant(), pins.DC_PINS), f"{mutant.__name__} slipped through"
+
+
+class MultSwapped(NumpyImpl):
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        return super().global_update_mult(grads, w, v, lr, momentum, wd, offsets, wd_mult, lr_mult)
+
+
+class MultOffByOneTensor(NumpyImpl):
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        return super().global_update_mult(grads, w, v, lr, momentum, wd, offsets, np.roll(lr_mult, 1), np.roll(wd_mult, 1))
+
+
+class MultOnVelocityToo(NumpyImpl):
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        wn, vn, wp = super().global_update_mult(grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult)
+        scale = np.empty_like(w)
+        for t, (a, b) in enumerate(zip(offsets[:-1], offsets[1:])):
+            scale[a:b] = lr_mult[t]
+        return w + scale * vn, vn, wp
+
+
+class DcasgdBackupNotRefreshed(NumpyImpl):
+    def dcasgd_step_c(self, g, w, bak, lr, lam):
+        return self.local_update_dc_c(w, g, bak, lr, lam), bak.copy()
+
+    def dcasgd_step_a(self, g, w, bak, ms, lr, lam, m, eps):
+        wn, msn = self.local_update_dc_a(w, g, bak, ms, lr, lam, m, eps)
+        return wn, bak.copy(), msn
+
+
+class DcasgdRolesSwapped(NumpyImpl):
+    def dcasgd_step_c(self, g, w, bak, lr, lam):
+        wn = w - F32(lr) * (g + (F32(lam) * (g * g)) * (bak - w))
+        return wn, wn.copy()
+
+
+@pytest.mark.parametrize("mutant", [MultSwapped, MultOffByOneTensor, MultOnVelocityToo, DcasgdBackupNotRefreshed,
+                                    DcasgdRolesSwapped], ids=lambda c: c.__name__)
+def test_planted_ext_mistake_is_caught(mutant):
+    assert _rejected_by(mutant(), pins.EXT_PINS), f"{mutant.__name__} slipped through"
 
 
 def test_round_to_f32_is_correctly_rounded():
