@@ -197,15 +197,80 @@ int odsgd_set_wd(odsgd_ctx* ctx, float wd);
 /*
  * Chooses the local update rule (Section 3.3).  ODSGD_LOCAL_SGD ignores the other
  * arguments.  ODSGD_LOCAL_DC_C uses `lambda` (Eq. 4).  ODSGD_LOCAL_DC_A uses `lambda`,
- * the mean-square decay `m` and `eps` (Eq. 5, Eq. 6) and needs one mean-square arena
- * per worker with a local buffer: `mean_square` is a host array of n_workers device
- * pointers (n_params floats each, caller-owned and caller-initialised, normally zeros);
- * pass NULL for the other rules.  In both delay-compensated rules the vector the
+ * the mean-square decay `m` and `eps` (Eq. 5, Eq. 6); a local update under this rule needs
+ * one mean-square arena for the worker it updates: `mean_square` is a host array of
+ * n_workers device pointers (n_params floats each, caller-owned and caller-initialised,
+ * normally zeros; entries may be NULL for workers that are never updated locally, and the
+ * whole table may be NULL when the rule is only used by odsgd_dcasgd_step); pass NULL for
+ * the other rules.  A local update of a worker without its arena fails with ERR_STATE.  In both delay-compensated rules the vector the
  * gradient was computed on (the paper's w_t) is the worker's previous local weights,
  * i.e. the content of local[worker] before the call, which is then overwritten.
  */
 int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float eps,
                          float* const* mean_square);
+
+/*
+ * Per-tensor multipliers of the stock updater the paper relies on (Section 3.3: the global
+ * updater is the framework's own): tensor t is updated with lr * lr_mult[t] and
+ * wd * wd_mult[t] (each product rounded once), e.g. wd_mult = 0 for biases and batch-norm
+ * scales.  `lr_mult`, `wd_mult`: HOST arrays of n_tensors floats; NULL means all ones; both
+ * NULL switches the feature off.  The library keeps a small device table (offsets and the two
+ * multiplier arrays, 16 bytes per tensor), allocated by this call with cudaMalloc and filled by
+ * a copy enqueued on `stream`; it is freed by odsgd_destroy or when the feature is switched
+ * off.  Applies to the global, fused and SSGD calls; the ASGD and local rules are unaffected.
+ * The 128-bit kernels need every tensor offset to be a multiple of 4 elements; otherwise the
+ * call fails with ERR_ALIGN unless ODSGD_FLAG_ALLOW_UNALIGNED is set (scalar kernel).
+ * Errors: ERR_CUDA (allocation or copy failed), ERR_ALIGN.
+ */
+int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const float* wd_mult, void* stream);
+
+/*
+ * DC-ASGD at the parameter server (the paper's fourth comparison algorithm, Section 4.1):
+ * Eq. 4 or Eq. 5/6 applied to one arriving gradient, with the current global weights in the
+ * role of w_{t+tau} and local[worker_id] - the copy worker `worker_id` pulled last - in the
+ * role of w_t:
+ *     w <- w - lr * (g + lambda' * g*g * (w - local[worker_id]));   local[worker_id] <- w
+ * (the worker pulls the new weights).  lambda, m, eps come from odsgd_set_local_rule(), whose
+ * rule must be ODSGD_LOCAL_DC_C or ODSGD_LOCAL_DC_A; for DC_A the server's single running mean
+ * square lives in the arena given to odsgd_set_server_mean_square().  No momentum, no weight
+ * decay (Eq. 4/5 have neither).  In place on the current weights; like the ASGD step it
+ * invalidates the backup weights.  local[worker_id] must hold the weights that worker pulled
+ * (initially a copy of w_0).
+ * Errors: ERR_STATE (rule is SGD, or DC_A without a server mean-square arena), ERR_ARG, ERR_OVERLAP.
+ */
+int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream);
+
+/* Device arena (n_params floats, caller-owned, normally zero-filled) for Eq. 6's state at the server. */
+int odsgd_set_server_mean_square(odsgd_ctx* ctx, float* mean_square);
+
+/*
+ * The worker loop of Algorithm 2 as a state machine.  odsgd_set_warmup() sets wp, the number
+ * of warm-up iterations (the paper uses 200 iterations, or 0-5 epochs); it may be called
+ * only before the first odsgd_step().  odsgd_step() runs iteration k = 0, 1, 2, ...:
+ *   k <  wp : SSGD step (warm-up stage: workers wait for and train on the new weights);
+ *   k >= wp : fused global + local update for every worker that has a local buffer (at
+ *             k = wp, the last warm-up iteration of Algorithm 2, the gradient was still taken
+ *             on the global weights, so the delay-compensated rules see no delay there).
+ * The copy "w_bak = w_t" of iteration wp - 1 is implicit: the backup is the weight half the
+ * update reads.  odsgd_get_train_weights() tells which arena worker `worker_id` computes its
+ * next gradient on: the current global weights while the next iteration index is <= wp, its
+ * local arena afterwards.
+ */
+int odsgd_set_warmup(odsgd_ctx* ctx, uint64_t wp);
+int odsgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream);
+int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights);
+
+/*
+ * Learning-rate schedules the paper's runs use (Section 4): host-side helpers that return the
+ * rate for iteration `step`; feed the result to odsgd_set_lr / odsgd_set_local_lr.
+ *   step decay : base * factor^(number of boundaries <= step)       (divide by 10 at given epochs)
+ *   linear ramp: start + (end - start) * min(step, ramp) / ramp     (the "WP" ramp 0.1 -> 0.8)
+ *   polynomial : end + (base - end) * (1 - min(step, total)/total)^power   (power 2 in the paper)
+ * Computed in double, rounded once to float.
+ */
+float odsgd_lr_step_decay(float base_lr, float factor, const uint64_t* boundaries, size_t n_boundaries, uint64_t step);
+float odsgd_lr_linear_ramp(float start_lr, float end_lr, uint64_t ramp_steps, uint64_t step);
+float odsgd_lr_poly_decay(float base_lr, float end_lr, float power, uint64_t total_steps, uint64_t step);
 
 /* Current and backup (one step old) weight arenas; either output pointer may be NULL.
  * *delayed is NULL when the context keeps no backup or none is valid yet. */

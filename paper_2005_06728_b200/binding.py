@@ -31,6 +31,9 @@ EXPORTS = (
     "odsgd_asgd_step", "odsgd_set_lr", "odsgd_set_local_lr", "odsgd_set_momentum", "odsgd_set_wd",
     "odsgd_set_local_rule", "odsgd_get_weights", "odsgd_get_step", "odsgd_set_step",
     "odsgd_set_launch_config", "odsgd_get_launch_count", "odsgd_last_error",
+    "odsgd_set_tensor_multipliers", "odsgd_dcasgd_step", "odsgd_set_server_mean_square", "odsgd_set_warmup",
+    "odsgd_step", "odsgd_get_train_weights", "odsgd_lr_step_decay", "odsgd_lr_linear_ramp",
+    "odsgd_lr_poly_decay",
 )
 
 
@@ -89,6 +92,15 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_set_launch_config": ([vp, ci, ci], ci),
         "odsgd_get_launch_count": ([vp, u64p], ci),
         "odsgd_last_error": ([vp], ctypes.c_char_p),
+        "odsgd_set_tensor_multipliers": ([vp, ctypes.POINTER(cf), ctypes.POINTER(cf), vp], ci),
+        "odsgd_dcasgd_step": ([vp, ci, vp, vp], ci),
+        "odsgd_set_server_mean_square": ([vp, vp], ci),
+        "odsgd_set_warmup": ([vp, ctypes.c_uint64], ci),
+        "odsgd_step": ([vp, pvp, vp], ci),
+        "odsgd_get_train_weights": ([vp, ci, ctypes.POINTER(vp)], ci),
+        "odsgd_lr_step_decay": ([cf, cf, u64p, ctypes.c_size_t, ctypes.c_uint64], cf),
+        "odsgd_lr_linear_ramp": ([cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
+        "odsgd_lr_poly_decay": ([cf, cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
     }
     for name, (argtypes, restype) in sig.items():
         fn = getattr(lib, name)  # AttributeError if the library lacks a declared symbol
@@ -161,6 +173,9 @@ class Odsgd:
             raise OdsgdError(rc, msg)
         self._device = w_a.device
         self._by_ptr = {t.data_ptr(): t for t in (w_a, w_b, w_delayed) if t is not None}
+        if local is not None:
+            self._by_ptr.update({t.data_ptr(): t for t in local if t is not None})
+        self.n_tensors = len(offs) - 1
 
     # -- plumbing
     def _check(self, rc: int) -> None:
@@ -223,6 +238,39 @@ class Odsgd:
     def asgd_step(self, worker_id: int, grad: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
         self._check(self._lib.odsgd_asgd_step(self._h, worker_id, _dev_ptr(grad, "grad", self.n_params),
                                               _stream_handle(stream)))
+
+    def dcasgd_step(self, worker_id: int, grad: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+        self._check(self._lib.odsgd_dcasgd_step(self._h, worker_id, _dev_ptr(grad, "grad", self.n_params),
+                                                _stream_handle(stream)))
+
+    def step_update(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
+        """odsgd_step: one iteration of Algorithm 2's state machine (warm-up SSGD, then OD-SGD)."""
+        self._check(self._lib.odsgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
+        self._bound = list(grads)
+
+    def set_warmup(self, wp: int) -> None:
+        self._check(self._lib.odsgd_set_warmup(self._h, wp))
+
+    def train_weights(self, worker_id: int) -> torch.Tensor:
+        """The tensor worker `worker_id` computes its next gradient on."""
+        p = ctypes.c_void_p()
+        self._check(self._lib.odsgd_get_train_weights(self._h, worker_id, ctypes.byref(p)))
+        return self._by_ptr[p.value]
+
+    def set_tensor_multipliers(self, lr_mult: Optional[Sequence[float]], wd_mult: Optional[Sequence[float]],
+                               stream: Optional[torch.cuda.Stream] = None) -> None:
+        def arr(x):
+            if x is None:
+                return None
+            if len(x) != self.n_tensors:
+                raise ValueError(f"need {self.n_tensors} multipliers, got {len(x)}")
+            return (ctypes.c_float * len(x))(*[float(t) for t in x])
+
+        self._check(self._lib.odsgd_set_tensor_multipliers(self._h, arr(lr_mult), arr(wd_mult), _stream_handle(stream)))
+
+    def set_server_mean_square(self, ms: Optional[torch.Tensor]) -> None:
+        self._check(self._lib.odsgd_set_server_mean_square(self._h, _dev_ptr(ms, "mean_square", self.n_params)))
+        self._keep.append(ms)
 
     # -- settings
     def set_lr(self, lr: float) -> None:
@@ -316,3 +364,24 @@ def odsgd_ssgd_step(ctx: Odsgd, worker_grads, stream=None) -> None:
 
 def odsgd_asgd_step(ctx: Odsgd, worker_id: int, grad, stream=None) -> None:
     ctx.asgd_step(worker_id, grad, stream)
+
+
+def odsgd_dcasgd_step(ctx: Odsgd, worker_id: int, grad, stream=None) -> None:
+    ctx.dcasgd_step(worker_id, grad, stream)
+
+
+def odsgd_step(ctx: Odsgd, worker_grads, stream=None) -> None:
+    ctx.step_update(worker_grads, stream)
+
+
+def odsgd_lr_step_decay(base_lr: float, factor: float, boundaries: Sequence[int], step: int) -> float:
+    b = (ctypes.c_uint64 * len(boundaries))(*[int(x) for x in boundaries])
+    return load_library().odsgd_lr_step_decay(base_lr, factor, b, len(boundaries), step)
+
+
+def odsgd_lr_linear_ramp(start_lr: float, end_lr: float, ramp_steps: int, step: int) -> float:
+    return load_library().odsgd_lr_linear_ramp(start_lr, end_lr, ramp_steps, step)
+
+
+def odsgd_lr_poly_decay(base_lr: float, end_lr: float, power: float, total_steps: int, step: int) -> float:
+    return load_library().odsgd_lr_poly_decay(base_lr, end_lr, power, total_steps, step)

@@ -3,6 +3,7 @@
 // allocation of parameter-sized memory, no synchronisation.
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -38,6 +39,13 @@ struct odsgd_ctx {
     uint64_t launches = 0;
     int block_threads = 0;  // 0 = built-in
     int ctas_per_sm = 0;    // 0 = built-in
+    // per-tensor multipliers: one device allocation [offsets u64 x (T+1) | lr_mult f32 x T | wd_mult f32 x T]
+    void* table_dev = nullptr;
+    std::vector<unsigned char> table_host;  // staging copy the upload reads from
+    bool mult_on = false;
+    float* server_ms = nullptr;  // Eq. 6 state of the server-side DC-ASGD step
+    uint64_t wp = 0;             // Algorithm 2's warm-up length
+    uint64_t iter = 0;           // iterations done through odsgd_step
     std::string err;
 };
 
@@ -87,6 +95,7 @@ std::vector<Named> state_buffers(const odsgd_ctx* c) {
         if (c->local[m]) s.push_back({c->local[m], "local", m});
         if (c->mean_square[m]) s.push_back({c->mean_square[m], "mean_square", m});
     }
+    if (c->server_ms) s.push_back({c->server_ms, "server_mean_square", -1});
     return s;
 }
 
@@ -150,10 +159,10 @@ int too_wide(odsgd_ctx* c, int block) {
     return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
 }
 
-template <bool DET, int NL, int LOCAL, int RULE>
-int launch_server_t(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
+int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
-    auto kernel = server_kernel<DET, NL, LOCAL, RULE>;
+    auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT>;
     static int cached_block = 0, cached_res = 0;
     if (cached_block != block) {
         cached_res = resident_ctas(kernel, block);
@@ -163,6 +172,12 @@ int launch_server_t(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
     const int grid = grid_for(c, a.n, NL, block, kUnroll, kServerCtasPerSm);
     kernel<<<grid, block, 0, st>>>(a);
     return after_launch(c, "server kernel launch");
+}
+
+template <bool DET, int NL, int LOCAL, int RULE>
+int launch_server_t(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+    return c->mult_on ? launch_server_m<DET, NL, LOCAL, RULE, true>(c, a, st)
+                      : launch_server_m<DET, NL, LOCAL, RULE, false>(c, a, st);
 }
 
 template <bool DET, int NL, int LOCAL>
@@ -190,10 +205,10 @@ int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, 
     return lanes == 4 ? launch_server_l<false, 4>(c, a, local_mode, st) : launch_server_l<false, 1>(c, a, local_mode, st);
 }
 
-template <bool DET, int NL, int RULE>
+template <bool DET, int NL, int RULE, bool SERVER>
 int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
-    auto kernel = local_kernel<DET, NL, RULE>;
+    auto kernel = local_kernel<DET, NL, RULE, SERVER>;
     static int cached_block = 0, cached_res = 0;
     if (cached_block != block) {
         cached_res = resident_ctas(kernel, block);
@@ -205,18 +220,22 @@ int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
 }
 
 template <bool DET, int NL>
-int launch_local_r(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
+int launch_local_r(odsgd_ctx* c, const LocalArgs& a, bool server, cudaStream_t st) {
+    if (server) {  // DC-ASGD at the server: only the delay-compensated rules exist there
+        return c->local_rule == ODSGD_LOCAL_DC_C ? launch_local_t<DET, NL, ODSGD_LOCAL_DC_C, true>(c, a, st)
+                                                 : launch_local_t<DET, NL, ODSGD_LOCAL_DC_A, true>(c, a, st);
+    }
     switch (c->local_rule) {
-        case ODSGD_LOCAL_SGD: return launch_local_t<DET, NL, ODSGD_LOCAL_SGD>(c, a, st);
-        case ODSGD_LOCAL_DC_C: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_C>(c, a, st);
-        default: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_A>(c, a, st);
+        case ODSGD_LOCAL_SGD: return launch_local_t<DET, NL, ODSGD_LOCAL_SGD, false>(c, a, st);
+        case ODSGD_LOCAL_DC_C: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_C, false>(c, a, st);
+        default: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_A, false>(c, a, st);
     }
 }
 
-int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, cudaStream_t st) {
+int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, bool server, cudaStream_t st) {
     const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
-    if (det) return lanes == 4 ? launch_local_r<true, 4>(c, a, st) : launch_local_r<true, 1>(c, a, st);
-    return lanes == 4 ? launch_local_r<false, 4>(c, a, st) : launch_local_r<false, 1>(c, a, st);
+    if (det) return lanes == 4 ? launch_local_r<true, 4>(c, a, server, st) : launch_local_r<true, 1>(c, a, server, st);
+    return lanes == 4 ? launch_local_r<false, 4>(c, a, server, st) : launch_local_r<false, 1>(c, a, server, st);
 }
 
 template <bool DET, int NL>
@@ -246,6 +265,7 @@ LocalParams local_params(const odsgd_ctx* c) {
     p.m = c->dc_m;
     p.one_minus_m = 1.0f - c->dc_m;
     p.eps = c->dc_eps;
+    p.first = 0;
     return p;
 }
 
@@ -298,7 +318,8 @@ int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mo
 // Shared body of the global, fused and SSGD calls.
 //   keep_backup: OD-SGD server step (the old weights stay available to the workers)
 //   local_id:    -2 none, -1 all workers, >= 0 one worker
-int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, void* stream) {
+int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, void* stream,
+                bool first_delayed_step = false) {
     if (!c) return ODSGD_ERR_ARG;
     std::vector<Named> ptrs;
     int rc = check_grads(c, grads, &ptrs);
@@ -315,6 +336,15 @@ int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
     a.momentum = c->momentum;
     a.wd = c->wd;
     a.lp = local_params(c);
+    a.lp.first = first_delayed_step ? 1 : 0;
+    if (c->mult_on) {
+        const size_t nt = c->offsets.size() - 1;
+        unsigned char* base = static_cast<unsigned char*>(c->table_dev);
+        a.t_off = reinterpret_cast<const unsigned long long*>(base);
+        a.t_lr_mult = reinterpret_cast<const float*>(base + (nt + 1) * sizeof(unsigned long long));
+        a.t_wd_mult = a.t_lr_mult + nt;
+        a.n_tensors = (unsigned int)nt;
+    }
     a.w_in = c->w[c->cur];
     const float* delayed_after = nullptr;
     int next_cur = c->cur;
@@ -339,8 +369,14 @@ int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
         rc = bind_local_outputs(c, local_id, &a, &local_mode, &ptrs);
         if (rc != ODSGD_OK) return rc;
     }
-    const int lanes = lanes_for(c, ptrs);
+    int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
+    if (c->mult_on && lanes == 4) {
+        // a 128-bit vector must not straddle two tensors (set_tensor_multipliers has checked that
+        // the scalar path is allowed when it would)
+        for (size_t o : c->offsets)
+            if (o % 4 != 0) { lanes = 1; break; }
+    }
 
     rc = launch_server(c, a, lanes, local_mode, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
@@ -437,6 +473,7 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
 
 int odsgd_destroy(odsgd_ctx* ctx) {
     if (!ctx) return ODSGD_ERR_ARG;
+    if (ctx->table_dev) cudaFree(ctx->table_dev);
     delete ctx;
     return ODSGD_OK;
 }
@@ -469,13 +506,14 @@ int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     a.g = c->bound[worker_id];
     a.x = c->local[worker_id];
     a.ms = c->mean_square[worker_id];
+    a.w_out = nullptr;
     a.n = c->n;
     a.lp = local_params(c);
     std::vector<Named> ptrs = {{a.w_bak, "w_delayed", -1}, {a.g, "worker_grads", worker_id}, {a.x, "local", worker_id}};
     if (need_ms) ptrs.push_back({a.ms, "mean_square", worker_id});
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
-    return launch_local(c, a, lanes, static_cast<cudaStream_t>(stream));
+    return launch_local(c, a, lanes, false, static_cast<cudaStream_t>(stream));
 }
 
 int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging, int worker_id,
@@ -562,16 +600,13 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
     odsgd_ctx* c = ctx;
     if (rule != ODSGD_LOCAL_SGD && rule != ODSGD_LOCAL_DC_C && rule != ODSGD_LOCAL_DC_A)
         return fail(c, ODSGD_ERR_ARG, "unknown local rule");
-    if (rule == ODSGD_LOCAL_DC_A) {
-        if (!mean_square) return fail(c, ODSGD_ERR_ARG, "ODSGD_LOCAL_DC_A needs mean_square arenas");
+    if (rule == ODSGD_LOCAL_DC_A && mean_square) {
         odsgd_ctx probe = *c;
         for (int w = 0; w < c->n_workers; ++w) probe.mean_square[w] = mean_square[w];
         const std::vector<Named> st = state_buffers(&probe);
         const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
-        for (int w = 0; w < c->n_workers; ++w) {
-            if (c->local[w] && !mean_square[w]) return fail(c, ODSGD_ERR_ARG, "mean_square[" + std::to_string(w) + "] is NULL");
+        for (int w = 0; w < c->n_workers; ++w)
             if (mean_square[w] && !aligned(mean_square[w], need)) return fail(c, ODSGD_ERR_ALIGN, "mean_square arena misaligned");
-        }
         const int rc = check_distinct(c, st, c->n * sizeof(float));
         if (rc != ODSGD_OK) return rc;
         for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = mean_square[w];
@@ -583,6 +618,152 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
     c->dc_m = m;
     c->dc_eps = eps;
     return ODSGD_OK;
+}
+
+int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const float* wd_mult, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (!lr_mult && !wd_mult) {
+        if (c->table_dev) cudaFree(c->table_dev);
+        c->table_dev = nullptr;
+        c->mult_on = false;
+        return ODSGD_OK;
+    }
+    const size_t nt = c->offsets.size() - 1;
+    if (!(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED))
+        for (size_t o : c->offsets)
+            if (o % 4 != 0)
+                return fail(c, ODSGD_ERR_ALIGN, "tensor offset " + std::to_string(o) + " is not a multiple of 4 elements (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
+    const size_t bytes = (nt + 1) * sizeof(unsigned long long) + 2 * nt * sizeof(float);
+    c->table_host.resize(bytes);
+    unsigned long long* off = reinterpret_cast<unsigned long long*>(c->table_host.data());
+    float* lm = reinterpret_cast<float*>(c->table_host.data() + (nt + 1) * sizeof(unsigned long long));
+    float* wm = lm + nt;
+    for (size_t t = 0; t <= nt; ++t) off[t] = c->offsets[t];
+    for (size_t t = 0; t < nt; ++t) {
+        lm[t] = lr_mult ? lr_mult[t] : 1.0f;
+        wm[t] = wd_mult ? wd_mult[t] : 1.0f;
+    }
+    if (!c->table_dev) {
+        const cudaError_t e = cudaMalloc(&c->table_dev, bytes);
+        if (e != cudaSuccess) {
+            c->table_dev = nullptr;
+            return fail(c, ODSGD_ERR_CUDA, std::string("multiplier table allocation: ") + cudaGetErrorString(e));
+        }
+    }
+    const cudaError_t e = cudaMemcpyAsync(c->table_dev, c->table_host.data(), bytes, cudaMemcpyHostToDevice,
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("multiplier table upload: ") + cudaGetErrorString(e));
+    c->mult_on = true;
+    return ODSGD_OK;
+}
+
+int odsgd_set_server_mean_square(odsgd_ctx* ctx, float* mean_square) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (mean_square) {
+        const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
+        if (!aligned(mean_square, need)) return fail(c, ODSGD_ERR_ALIGN, "server mean-square arena misaligned");
+        const size_t bytes = c->n * sizeof(float);
+        float* keep = c->server_ms;
+        c->server_ms = nullptr;
+        for (const Named& s : state_buffers(c))
+            if (overlap(mean_square, s.p, bytes)) {
+                c->server_ms = keep;
+                return fail(c, ODSGD_ERR_OVERLAP, "server mean-square arena overlaps " + label(s));
+            }
+    }
+    c->server_ms = mean_square;
+    return ODSGD_OK;
+}
+
+int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (!grad) return fail(c, ODSGD_ERR_ARG, "grad is NULL");
+    if (c->local_rule != ODSGD_LOCAL_DC_C && c->local_rule != ODSGD_LOCAL_DC_A)
+        return fail(c, ODSGD_ERR_STATE, "choose ODSGD_LOCAL_DC_C or ODSGD_LOCAL_DC_A with odsgd_set_local_rule first");
+    if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no backup (local) buffer for worker " + std::to_string(worker_id));
+    const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
+    if (need_ms && !c->server_ms) return fail(c, ODSGD_ERR_STATE, "ODSGD_LOCAL_DC_A at the server needs odsgd_set_server_mean_square");
+    const size_t bytes = c->n * sizeof(float);
+    const Named g{grad, "grad", -1};
+    for (const Named& s : state_buffers(c))
+        if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, "grad overlaps " + label(s));
+    LocalArgs a;
+    a.w_bak = c->w[c->cur];
+    a.w_out = c->w[c->cur];
+    a.g = grad;
+    a.x = c->local[worker_id];
+    a.ms = c->server_ms;
+    a.n = c->n;
+    a.lp = local_params(c);
+    a.lp.local_lr = c->lr;  // the server applies its own learning rate
+    std::vector<Named> ptrs = {g, {a.w_out, "w", -1}, {a.x, "local", worker_id}};
+    if (need_ms) ptrs.push_back({a.ms, "server_mean_square", -1});
+    const int lanes = lanes_for(c, ptrs);
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+    const int rc = launch_local(c, a, lanes, true, static_cast<cudaStream_t>(stream));
+    if (rc != ODSGD_OK) return rc;
+    c->step += 1;
+    c->grads_bound = false;
+    c->delayed = nullptr;
+    return ODSGD_OK;
+}
+
+int odsgd_set_warmup(odsgd_ctx* ctx, uint64_t wp) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (ctx->iter != 0) return fail(ctx, ODSGD_ERR_STATE, "the warm-up length can only be set before the first odsgd_step");
+    ctx->wp = wp;
+    return ODSGD_OK;
+}
+
+int odsgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    int rc;
+    if (c->iter < c->wp) {
+        rc = server_call(c, worker_grads, false, -2, stream);  // warm-up stage: SSGD
+    } else {
+        // from the last warm-up iteration on: server step + local update of every worker; at
+        // iteration wp itself the gradients were taken on the global weights (no delay yet)
+        rc = server_call(c, worker_grads, true, -1, stream, c->iter == c->wp);
+    }
+    if (rc == ODSGD_OK) c->iter += 1;
+    return rc;
+}
+
+int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights) {
+    if (!ctx || !weights) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (c->iter <= c->wp) {
+        *weights = c->w[c->cur];
+        return ODSGD_OK;
+    }
+    if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
+    *weights = c->local[worker_id];
+    return ODSGD_OK;
+}
+
+float odsgd_lr_step_decay(float base_lr, float factor, const uint64_t* boundaries, size_t n_boundaries, uint64_t step) {
+    double lr = base_lr;
+    for (size_t i = 0; i < n_boundaries; ++i)
+        if (boundaries && boundaries[i] <= step) lr *= (double)factor;
+    return (float)lr;
+}
+
+float odsgd_lr_linear_ramp(float start_lr, float end_lr, uint64_t ramp_steps, uint64_t step) {
+    if (ramp_steps == 0 || step >= ramp_steps) return end_lr;
+    const double f = (double)step / (double)ramp_steps;
+    return (float)((double)start_lr + ((double)end_lr - (double)start_lr) * f);
+}
+
+float odsgd_lr_poly_decay(float base_lr, float end_lr, float power, uint64_t total_steps, uint64_t step) {
+    if (total_steps == 0 || step >= total_steps) return end_lr;
+    const double f = 1.0 - (double)step / (double)total_steps;
+    return (float)((double)end_lr + ((double)base_lr - (double)end_lr) * pow(f, (double)power));
 }
 
 int odsgd_get_weights(odsgd_ctx* ctx, float** current, float** delayed) {

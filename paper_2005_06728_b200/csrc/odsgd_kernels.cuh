@@ -64,6 +64,7 @@ struct LocalParams {
     float m;            // Eq. 6 decay
     float one_minus_m;  // computed once on the host in fp32
     float eps;          // Eq. 5
+    int first;          // 1: the gradient was computed on w_bak itself (first delayed step), x_prev := w_bak
 };
 
 // Kernel argument block, passed by value (constant bank): no dependent device
@@ -82,13 +83,19 @@ struct ServerArgs {
     float inv_n;                        // 1.0f / n_workers, computed on the host
     float lr, momentum, wd;
     LocalParams lp;
+    // per-tensor multipliers (MULT kernels only): device table, n_tensors + 1 ascending offsets
+    const unsigned long long* t_off;
+    const float* t_lr_mult;
+    const float* t_wd_mult;
+    unsigned int n_tensors;
 };
 
 struct LocalArgs {
     const float* w_bak;
     const float* g;
-    float* x;   // read (previous local weights) by the delay-compensated rules, then written
-    float* ms;  // Eq. 6 state or null
+    float* x;      // read (previous local weights) by the delay-compensated rules, then written
+    float* ms;     // Eq. 6 state or null
+    float* w_out;  // server-side DC-ASGD only: the global weights, which receive the result too
     unsigned long long n;
     LocalParams lp;
 };
@@ -206,13 +213,35 @@ __device__ __forceinline__ float local_rule(float w_bak, float g, float x_prev, 
     return O::sub(w_bak, O::mul(p.local_lr, O::add(g, comp)));  // Eq. 4 / Eq. 5
 }
 
+// ------------------------------------------------------------------ per-tensor multipliers
+// Which tensor an element belongs to: binary search over the offset table (a few hundred
+// entries at most, L1/L2 resident), skipped while the thread stays inside the tensor it
+// found last (the large tensors hold almost all elements).
+struct TensorCursor {
+    unsigned long long lo = 1, hi = 0;  // empty range: the first lookup searches
+    float lr_mult = 1.0f, wd_mult = 1.0f;
+};
+
+__device__ __forceinline__ void find_tensor(const ServerArgs& a, unsigned long long off, TensorCursor& c) {
+    if (off >= c.lo && off < c.hi) return;
+    unsigned int lo = 0, hi = a.n_tensors;  // t_off[lo] <= off < t_off[hi]
+    while (hi - lo > 1) {
+        const unsigned int mid = (lo + hi) >> 1;
+        if (__ldg(a.t_off + mid) <= off) lo = mid; else hi = mid;
+    }
+    c.lo = __ldg(a.t_off + lo);
+    c.hi = __ldg(a.t_off + lo + 1);
+    c.lr_mult = __ldg(a.t_lr_mult + lo);
+    c.wd_mult = __ldg(a.t_wd_mult + lo);
+}
+
 // ------------------------------------------------------------------ server kernel
 // One vector (NL lanes) of the arena at element offset `off`:
 // sum the workers in order, apply the server rule, and (LOCAL != none) the
 // local rule for one worker or for every worker that has a local buffer.
-template <bool DET, int NL, int LOCAL, int RULE, int U>
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int U>
 __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsigned long long (&off)[U],
-                                               const bool (&ok)[U]) {
+                                               const bool (&ok)[U], TensorCursor& cur) {
     using O = Op<DET>;
     Vec<NL> w[U], v[U], s[U], gl[U];
 #pragma unroll
@@ -257,7 +286,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                             float* xp = a.x[m];
                             if (xp != nullptr) {
                                 Vec<NL> xo, xv, msv;
-                                if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(xp + off[u]);
+                                if (RULE != ODSGD_LOCAL_SGD) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
                                 if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[m] + off[u]);
 #pragma unroll
                                 for (int l = 0; l < NL; ++l) {
@@ -276,15 +305,21 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
     for (int u = 0; u < U; ++u) {
         if (!ok[u]) continue;
         Vec<NL> wn, vn;
+        float lr = a.lr, wd = a.wd;
+        if (MULT) {  // lr_t = lr * lr_mult[t], wd_t = wd * wd_mult[t], one rounding each
+            find_tensor(a, off[u], cur);
+            lr = O::mul(a.lr, cur.lr_mult);
+            wd = O::mul(a.wd, cur.wd_mult);
+        }
 #pragma unroll
         for (int l = 0; l < NL; ++l) {
             const float gbar = O::mul(s[u].e[l], a.inv_n);
-            server_rule<DET>(gbar, w[u].e[l], v[u].e[l], a.lr, a.momentum, a.wd, wn.e[l], vn.e[l]);
+            server_rule<DET>(gbar, w[u].e[l], v[u].e[l], lr, a.momentum, wd, wn.e[l], vn.e[l]);
         }
         if (LOCAL == kLocalOne) {
             float* xp = a.x[0];
             Vec<NL> xo, xv, msv;
-            if (RULE != ODSGD_LOCAL_SGD) xv = load_stream<NL>(xp + off[u]);
+            if (RULE != ODSGD_LOCAL_SGD) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
             if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[0] + off[u]);
 #pragma unroll
             for (int l = 0; l < NL; ++l) {
@@ -299,8 +334,9 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
     }
 }
 
-template <bool DET, int NL, int LOCAL, int RULE>
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
+    TensorCursor cur;
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * kUnroll;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
@@ -313,7 +349,7 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
             ok[u] = i < nvec;
             off[u] = i * NL;
         }
-        server_vectors<DET, NL, LOCAL, RULE, kUnroll>(a, off, ok);
+        server_vectors<DET, NL, LOCAL, RULE, MULT, kUnroll>(a, off, ok, cur);
     }
     if (NL > 1) {
         // ragged tail: the last n % NL elements, one lane each
@@ -321,7 +357,7 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
         if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
             const unsigned long long off1[1] = {done + threadIdx.x};
             const bool ok1[1] = {true};
-            server_vectors<DET, 1, LOCAL, RULE, 1>(a, off1, ok1);
+            server_vectors<DET, 1, LOCAL, RULE, MULT, 1>(a, off1, ok1, cur);
         }
     }
 }
@@ -330,16 +366,19 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
 // Few streams per element (2-4 reads, 1-2 writes): each thread takes kSmallUnroll vectors per
 // tile and issues all their loads before the first store, which is what a plain copy needs
 // to approach the copy ceiling of the part.
-template <bool DET, int NL, int RULE, int U>
+// SERVER = true is DC-ASGD at the parameter server (Eq. 4 / Eq. 5 applied to an arriving
+// gradient): w_bak is then the live global vector, read coherently and overwritten with the
+// result, and x is the worker's backup copy, which receives the same result (the worker pulls).
+template <bool DET, int NL, int RULE, bool SERVER, int U>
 __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned long long (&off)[U],
                                               const bool (&ok)[U]) {
     Vec<NL> w[U], g[U], xv[U], msv[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (ok[u]) {
-            w[u] = load_grad<NL>(a.w_bak + off[u]);
+            w[u] = SERVER ? load_stream<NL>(a.w_bak + off[u]) : load_grad<NL>(a.w_bak + off[u]);
             g[u] = load_grad<NL>(a.g + off[u]);
-            if (RULE != ODSGD_LOCAL_SGD) xv[u] = load_stream<NL>(a.x + off[u]);
+            if (RULE != ODSGD_LOCAL_SGD) xv[u] = a.lp.first ? w[u] : load_stream<NL>(a.x + off[u]);
             if (RULE == ODSGD_LOCAL_DC_A) msv[u] = load_stream<NL>(a.ms + off[u]);
         }
     }
@@ -350,11 +389,12 @@ __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned
 #pragma unroll
         for (int l = 0; l < NL; ++l) xo.e[l] = local_rule<DET, RULE>(w[u].e[l], g[u].e[l], xv[u].e[l], msv[u].e[l], a.lp);
         store_stream<NL>(a.x + off[u], xo);
+        if (SERVER) store_stream<NL>(a.w_out + off[u], xo);
         if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms + off[u], msv[u]);
     }
 }
 
-template <bool DET, int NL, int RULE>
+template <bool DET, int NL, int RULE, bool SERVER>
 __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
@@ -368,14 +408,14 @@ __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
             ok[u] = i < nvec;
             off[u] = i * NL;
         }
-        local_vectors<DET, NL, RULE, kSmallUnroll>(a, off, ok);
+        local_vectors<DET, NL, RULE, SERVER, kSmallUnroll>(a, off, ok);
     }
     if (NL > 1) {
         const unsigned long long done = nvec * NL;
         if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
             const unsigned long long off1[1] = {done + threadIdx.x};
             const bool ok1[1] = {true};
-            local_vectors<DET, 1, RULE, 1>(a, off1, ok1);
+            local_vectors<DET, 1, RULE, SERVER, 1>(a, off1, ok1);
         }
     }
 }

@@ -151,6 +151,54 @@ class GpuImpl(Impl):
         return self._local(w_bak, g, local_lr, binding.LOCAL_DC_A, x_prev=x_prev, ms=ms, lam=lam, m=m, eps=eps)
 
 
+    def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
+        self.bufs = []
+        wa, b0 = dev_arena(w)
+        va, b1 = dev_arena(v)
+        other, b2 = dev_arena(np.zeros(wa.numel(), np.float32))
+        self.bufs += [(b0, wa.numel()), (b1, wa.numel()), (b2, wa.numel())]
+        vec_ok = all(int(o) % 4 == 0 for o in offsets)
+        ctx = binding.Odsgd(wa, va, n_workers=len(grads), lr=lr, local_lr=0.0, momentum=momentum, wd=wd,
+                            w_b=other if self.pingpong else None, w_delayed=None if self.pingpong else other,
+                            tensor_offsets=[int(o) for o in offsets],
+                            flags=self.flags | (0 if vec_ok else binding.FLAG_ALLOW_UNALIGNED))
+        ctx.set_tensor_multipliers(list(map(float, lr_mult)), list(map(float, wd_mult)))
+        ctx.global_update(self._grads(grads))
+        self._done()
+        res = (ctx.weights().cpu().numpy().copy(), va.cpu().numpy().copy(),
+               ctx.delayed_weights().cpu().numpy().copy())
+        ctx.close()
+        return res
+
+    def _dcasgd(self, g, w, bak, rule, lr, lam, ms=None, m=0.0, eps=0.0):
+        self.bufs = []
+        n = np.asarray(w).size
+        wa, b0 = dev_arena(w)
+        va, b1 = dev_arena(np.zeros(n, np.float32))
+        bk, b2 = dev_arena(bak)
+        self.bufs += [(b0, n), (b1, n), (b2, n)]
+        ctx = binding.Odsgd(wa, va, n_workers=2, lr=lr, local_lr=123.0, momentum=0.9, wd=0.1,
+                            local=[None, bk], flags=self.flags)
+        ctx.set_local_rule(rule, lam, m, eps, None)
+        msd = None
+        if ms is not None:
+            msd, b3 = dev_arena(ms)
+            self.bufs.append((b3, n))
+            ctx.set_server_mean_square(msd)
+        ctx.dcasgd_step(1, self._grads([g])[0])
+        self._done()
+        res = (wa.cpu().numpy().copy(), bk.cpu().numpy().copy(),
+               msd.cpu().numpy().copy() if msd is not None else None)
+        ctx.close()
+        return res
+
+    def dcasgd_step_c(self, g, w, bak, lr, lam):
+        return self._dcasgd(g, w, bak, binding.LOCAL_DC_C, lr, lam)[:2]
+
+    def dcasgd_step_a(self, g, w, bak, ms, lr, lam, m, eps):
+        return self._dcasgd(g, w, bak, binding.LOCAL_DC_A, lr, lam, ms=ms, m=m, eps=eps)
+
+
 def same_bits(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     a = np.ascontiguousarray(a, dtype=np.float32)
     b = np.ascontiguousarray(b, dtype=np.float32)

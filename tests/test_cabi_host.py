@@ -146,3 +146,28 @@ def test_product_does_not_reach_for_the_oracle():
         if f.endswith((".py", ".cpp", ".h")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2005_06728_b200" not in text and "odsgd.h" not in text
+
+
+def test_lr_schedules_match_their_closed_forms(lib):
+    """Schedules named in the paper's Section 4: divide by 10 at given points, a linear ramp
+    (0.1 -> 0.8), polynomial decay with power 2."""
+    import numpy as np
+
+    f32 = np.float32
+    bounds = [80, 120]
+    for step, k in ((0, 0), (79, 0), (80, 1), (119, 1), (120, 2), (10_000, 2)):
+        assert binding.odsgd_lr_step_decay(0.1, 0.1, bounds, step) == f32(float(f32(0.1)) * float(f32(0.1)) ** k)
+    assert binding.odsgd_lr_step_decay(0.2, 0.1, [], 5) == f32(0.2)
+    s, e = float(f32(0.1)), float(f32(0.8))
+    for step in (0, 1, 250, 499, 500, 501, 10**9):
+        want = e if step >= 500 else s + (e - s) * step / 500
+        assert binding.odsgd_lr_linear_ramp(0.1, 0.8, 500, step) == f32(want)
+    assert binding.odsgd_lr_linear_ramp(0.1, 0.8, 0, 0) == f32(0.8)
+    b, e = float(f32(0.4)), float(f32(0.001))
+    for step in (0, 1, 1000, 89_999, 90_000, 100_000):
+        want = e if step >= 90_000 else e + (b - e) * (1 - step / 90_000) ** 2
+        assert binding.odsgd_lr_poly_decay(0.4, 0.001, 2.0, 90_000, step) == f32(want)
+    ramp = [binding.odsgd_lr_linear_ramp(0.1, 0.8, 100, k) for k in range(0, 120)]
+    assert all(a <= b for a, b in zip(ramp, ramp[1:])) and ramp[0] == f32(0.1) and ramp[-1] == f32(0.8)
+    poly = [binding.odsgd_lr_poly_decay(0.4, 0.0, 2.0, 100, k) for k in range(0, 120)]
+    assert all(a >= b for a, b in zip(poly, poly[1:])) and poly[-1] == 0.0
