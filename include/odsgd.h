@@ -225,6 +225,40 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
 int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const float* wd_mult, void* stream);
 
 /*
+ * Fused global + local update with per-tensor multipliers that never allocates.  (The paper
+ * has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * odsgd_set_tensor_multipliers() has to cudaMalloc a small device table.  Some callers must
+ * not do that: a server loop that runs beside training streams cannot afford cudaMalloc's
+ * device-wide synchronisation, and a process that has handed all device memory to its
+ * framework's pool may simply be refused.  For them this call does the same work as
+ * odsgd_set_tensor_multipliers(ctx, lr_mult, wd_mult, stream) followed by
+ * odsgd_fused_update(ctx, worker_grads, worker_id, stream), bit for bit, but keeps the table
+ * in a fixed array that is part of the library image: ODSGD_STATIC_TABLE_BYTES of device
+ * memory on every GPU that loads the library, held until the process exits.  It calls no
+ * cudaMalloc, no cudaFree and no allocating library routine, and does not touch the table of
+ * odsgd_set_tensor_multipliers() (which may be on or off; it is ignored here).
+ *
+ *   lr_mult, wd_mult  HOST arrays of n_tensors floats (NULL = all ones), read during the call
+ *   worker_id         0 .. n_workers-1, a worker that has a local buffer
+ *
+ * Limits: at most ODSGD_STATIC_MAX_TENSORS tensors (more: ERR_UNSUPPORTED, nothing is
+ * launched); local rule ODSGD_LOCAL_SGD only (else ERR_UNSUPPORTED); tensor offsets must be
+ * multiples of 4 elements unless ODSGD_FLAG_ALLOW_UNALIGNED is set (ERR_ALIGN).
+ * Set-up: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that first call outside any stream
+ * capture.  Sharing: every call on a device, from every context, writes the same array, and
+ * the array keeps the last call's table.  Each call rewrites all entries it uses before its
+ * kernel reads them, in stream order, so calls on ONE stream are safe back to back; calls
+ * whose work overlaps on the GPU (different streams, different threads) race on the array
+ * and must be serialised by the caller.
+ */
+#define ODSGD_STATIC_MAX_TENSORS 4096
+#define ODSGD_STATIC_TABLE_BYTES (16 * ODSGD_STATIC_MAX_TENSORS + 8)
+int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_grads, int worker_id,
+                                   const float* lr_mult, const float* wd_mult, void* stream);
+
+/*
  * DC-ASGD at the parameter server (the paper's fourth comparison algorithm, Section 4.1):
  * Eq. 4 or Eq. 5/6 applied to one arriving gradient, with the current global weights in the
  * role of w_{t+tau} and local[worker_id] - the copy worker `worker_id` pulled last - in the

@@ -33,7 +33,7 @@ EXPORTS = (
     "odsgd_set_launch_config", "odsgd_get_launch_count", "odsgd_last_error",
     "odsgd_set_tensor_multipliers", "odsgd_dcasgd_step", "odsgd_set_server_mean_square", "odsgd_set_warmup",
     "odsgd_step", "odsgd_get_train_weights", "odsgd_lr_step_decay", "odsgd_lr_linear_ramp",
-    "odsgd_lr_poly_decay",
+    "odsgd_lr_poly_decay", "odsgd_fused_update_mult_static",
 )
 
 
@@ -101,6 +101,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_lr_step_decay": ([cf, cf, u64p, ctypes.c_size_t, ctypes.c_uint64], cf),
         "odsgd_lr_linear_ramp": ([cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
         "odsgd_lr_poly_decay": ([cf, cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
+        "odsgd_fused_update_mult_static": ([vp, pvp, ci, ctypes.POINTER(cf), ctypes.POINTER(cf), vp], ci),
     }
     for name, (argtypes, restype) in sig.items():
         fn = getattr(lib, name)  # AttributeError if the library lacks a declared symbol
@@ -267,6 +268,25 @@ class Odsgd:
             return (ctypes.c_float * len(x))(*[float(t) for t in x])
 
         self._check(self._lib.odsgd_set_tensor_multipliers(self._h, arr(lr_mult), arr(wd_mult), _stream_handle(stream)))
+
+    def fused_update_mult_static(self, grads: Sequence[torch.Tensor], worker_id: int,
+                                 lr_mult: Optional[Sequence[float]], wd_mult: Optional[Sequence[float]],
+                                 stream: Optional[torch.cuda.Stream] = None) -> None:
+        """odsgd_fused_update_mult_static: the fused update with per-tensor multipliers for callers
+        that may not allocate device memory.  The multiplier table goes into a fixed array inside
+        the library instead of a cudaMalloc'ed one; all calls on a device share that array, so
+        calls whose GPU work could overlap must be serialised.  Make the first call on a device
+        outside any stream capture (it looks up the array's address)."""
+        def arr(x):
+            if x is None:
+                return None
+            if len(x) != self.n_tensors:
+                raise ValueError(f"need {self.n_tensors} multipliers, got {len(x)}")
+            return (ctypes.c_float * len(x))(*[float(t) for t in x])
+
+        self._check(self._lib.odsgd_fused_update_mult_static(self._h, self._grad_table(grads), worker_id,
+                                                             arr(lr_mult), arr(wd_mult), _stream_handle(stream)))
+        self._bound = list(grads)
 
     def set_server_mean_square(self, ms: Optional[torch.Tensor]) -> None:
         self._check(self._lib.odsgd_set_server_mean_square(self._h, _dev_ptr(ms, "mean_square", self.n_params)))

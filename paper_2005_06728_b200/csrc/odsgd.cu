@@ -801,6 +801,147 @@ int odsgd_get_launch_count(odsgd_ctx* ctx, uint64_t* launches) {
     return ODSGD_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Allocation-free variant of the fused update with per-tensor multipliers.
+//
+// Callers that may not cudaMalloc (a server loop that cannot take cudaMalloc's device-wide
+// synchronisation; a process whose device memory belongs to a framework pool) get the
+// multiplier table from g_static_table, a fixed array in the library image, instead of the
+// table odsgd_set_tensor_multipliers() allocates.  The name g_static_table is a device
+// symbol: host code must not pass it to a kernel as if it were an address.  Its device
+// address is looked up once per device with cudaGetSymbolAddress (static_table_address) and
+// that pointer is what the kernel receives.
+}  // extern "C"
+
+static __device__ __align__(256) unsigned char g_static_table[ODSGD_STATIC_TABLE_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_table_addr[kMaxDevices] = {};  // per device: address of g_static_table there
+unsigned char g_static_stage[ODSGD_STATIC_TABLE_BYTES];  // host copy the upload reads from (no allocation)
+
+// Device address of g_static_table on the current device; looked up on first use.
+int static_table_address(odsgd_ctx* c, unsigned char** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return fail(c, ODSGD_ERR_UNSUPPORTED, "device ordinal beyond the static table's bookkeeping");
+    if (dev != c->device) return fail(c, ODSGD_ERR_STATE, "the context was created on another device than the current one");
+    if (!g_static_table_addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_table);
+        if (e != cudaSuccess || !p) {
+            cudaGetLastError();
+            return fail(c, ODSGD_ERR_CUDA, std::string("cudaGetSymbolAddress(static table): ") + cudaGetErrorString(e));
+        }
+        g_static_table_addr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_static_table_addr[dev];
+    return ODSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_grads, int worker_id,
+                                   const float* lr_mult, const float* wd_mult, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
+    if (c->local_rule != ODSGD_LOCAL_SGD)
+        return fail(c, ODSGD_ERR_UNSUPPORTED, "the allocation-free call supports the ODSGD_LOCAL_SGD rule only");
+    const size_t nt = c->offsets.size() - 1;
+    if (nt > ODSGD_STATIC_MAX_TENSORS)
+        return fail(c, ODSGD_ERR_UNSUPPORTED, std::to_string(nt) + " tensors exceed the static table's limit of " +
+                                                  std::to_string(ODSGD_STATIC_MAX_TENSORS) +
+                                                  " (use odsgd_set_tensor_multipliers + odsgd_fused_update)");
+    bool vec_ok = true;
+    for (size_t o : c->offsets)
+        if (o % 4 != 0) vec_ok = false;
+    if (!vec_ok && !(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED))
+        return fail(c, ODSGD_ERR_ALIGN, "a tensor offset is not a multiple of 4 elements (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
+
+    std::vector<Named> ptrs;
+    int rc = check_grads(c, worker_grads, &ptrs);
+    if (rc != ODSGD_OK) return rc;
+    unsigned char* table = nullptr;
+    rc = static_table_address(c, &table);
+    if (rc != ODSGD_OK) return rc;
+
+    ServerArgs a;
+    memset(&a, 0, sizeof a);
+    for (int m = 0; m < c->n_workers; ++m) a.g[m] = worker_grads[m];
+    a.v = c->v;
+    a.n = c->n;
+    a.n_workers = c->n_workers;
+    a.inv_n = 1.0f / (float)c->n_workers;
+    a.lr = c->lr;
+    a.momentum = c->momentum;
+    a.wd = c->wd;
+    a.lp = local_params(c);
+    a.w_in = c->w[c->cur];
+    const float* delayed_after = nullptr;
+    int next_cur = c->cur;
+    if (c->pingpong) {
+        a.w_out = c->w[c->cur ^ 1];
+        delayed_after = c->w[c->cur];
+        next_cur = c->cur ^ 1;
+    } else {
+        a.w_out = c->w[c->cur];
+        if (c->w_delayed) {
+            a.w_prev = c->w_delayed;
+            delayed_after = c->w_delayed;
+        }
+    }
+    a.x[0] = c->local[worker_id];
+    a.local_worker = worker_id;
+    ptrs.push_back({a.w_in, "w", -1});
+    ptrs.push_back({a.w_out, "w", -1});
+    ptrs.push_back({a.v, "v", -1});
+    ptrs.push_back({a.x[0], "local", worker_id});
+    if (a.w_prev) ptrs.push_back({a.w_prev, "w_delayed", -1});
+    int lanes = lanes_for(c, ptrs);
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+    if (!vec_ok) lanes = 1;
+
+    // table layout: offsets u64 x (T+1) | lr_mult f32 x T | wd_mult f32 x T; every entry the
+    // kernel will read is rewritten here, so nothing depends on what an earlier call left
+    const size_t bytes = (nt + 1) * sizeof(unsigned long long) + 2 * nt * sizeof(float);
+    unsigned long long* off = reinterpret_cast<unsigned long long*>(g_static_stage);
+    float* lm = reinterpret_cast<float*>(g_static_stage + (nt + 1) * sizeof(unsigned long long));
+    float* wm = lm + nt;
+    for (size_t t = 0; t <= nt; ++t) off[t] = c->offsets[t];
+    for (size_t t = 0; t < nt; ++t) {
+        lm[t] = lr_mult ? lr_mult[t] : 1.0f;
+        wm[t] = wd_mult ? wd_mult[t] : 1.0f;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const cudaError_t e = cudaMemcpyAsync(table, g_static_stage, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("static table upload: ") + cudaGetErrorString(e));
+    a.t_off = reinterpret_cast<const unsigned long long*>(table);
+    a.t_lr_mult = reinterpret_cast<const float*>(table + (nt + 1) * sizeof(unsigned long long));
+    a.t_wd_mult = a.t_lr_mult + nt;
+    a.n_tensors = (unsigned int)nt;
+
+    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    if (det)
+        rc = lanes == 4 ? launch_server_m<true, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)
+                        : launch_server_m<true, 1, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st);
+    else
+        rc = lanes == 4 ? launch_server_m<false, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)
+                        : launch_server_m<false, 1, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st);
+    if (rc != ODSGD_OK) return rc;
+    c->cur = next_cur;
+    c->step += 1;
+    c->delayed = delayed_after;
+    c->grads_bound = true;
+    for (int m = 0; m < c->n_workers; ++m) c->bound[m] = worker_grads[m];
+    return ODSGD_OK;
+}
+
 const char* odsgd_last_error(odsgd_ctx* ctx) {
     return ctx ? ctx->err.c_str() : g_create_err.c_str();
 }
