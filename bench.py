@@ -50,7 +50,8 @@ def measured_traffic(step_bytes):
 
     try:
         note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_alexnet_m8.md")).read()
-        src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
+        src = b"".join(open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", f), "rb").read()
+                       for f in ("odsgd_kernels.cuh", "odsgd.cu"))
         ratio = float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1))
         sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1)
     except (OSError, AttributeError, ValueError):
@@ -75,6 +76,9 @@ def parse_args():
     ap.add_argument("--deterministic", action="store_true", help="time the one-rounding-per-operator flavour")
     ap.add_argument("--block", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
+    ap.add_argument("--multipliers", action="store_true", help="per-tensor lr/wd multipliers (no decay off the weight tensors)")
+    ap.add_argument("--local-rule", choices=["sgd", "dc_c", "dc_a"], default="sgd")
+    ap.add_argument("--all-locals", action="store_true", help="update every worker's local weights in the fused pass")
     ap.add_argument("--graph", type=int, default=0,
                     help="capture this many steps (even) in one CUDA graph and replay it; for the small, launch-bound sets")
     ap.add_argument("--no-e2e", action="store_true")
@@ -182,14 +186,16 @@ def run_cuda(args):
     M = args.workers or wl.n_workers
     n, P = wl.arena_len, wl.n_params
     free, total = torch.cuda.mem_get_info()
-    need = (M + 5) * n * 4
+    need = (M + 5 + (3 * M if args.all_locals else 0)) * n * 4
     if need > 0.9 * free:
         raise SystemExit(f"{wl.name} with {M} workers needs {need / 2**30:.1f} GiB; {free / 2**30:.1f} GiB free")
 
     w_a = W.make_weights(wl, dev)
     w_b = torch.zeros_like(w_a)
     v = W.make_momentum(wl, dev)
-    local = [torch.zeros_like(w_a)] + [None] * (M - 1)
+    n_locals = M if args.all_locals else 1
+    wid = -1 if args.all_locals else 0
+    local = [w_a.clone() for _ in range(n_locals)] + [None] * (M - n_locals)
     sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
     grads = [W.make_grad(wl, m, 0, dev, _sigma=sg, _pads=pads) for m in range(M)]
     flags = binding.FLAG_DETERMINISTIC if args.deterministic else 0
@@ -198,13 +204,21 @@ def run_cuda(args):
     if args.block or args.ctas_per_sm:
         ctx.set_launch_config(args.block, args.ctas_per_sm)
     stream = torch.cuda.current_stream()
+    extra_streams = 0  # arenas touched per local update beyond the plain rule's single store
+    if args.local_rule != "sgd":
+        rule = binding.LOCAL_DC_C if args.local_rule == "dc_c" else binding.LOCAL_DC_A
+        ms = [torch.zeros_like(w_a) for _ in range(n_locals)] + [None] * (M - n_locals) if rule == binding.LOCAL_DC_A else None
+        ctx.set_local_rule(rule, 0.04, 0.95, 1e-7, ms)
+        extra_streams = n_locals * (1 if rule == binding.LOCAL_DC_C else 3)  # x_prev read (+ mean square read, write)
+    if args.multipliers:
+        ctx.set_tensor_multipliers(None, [1.0 if t.kind == "weight" else 0.0 for t in wl.tensors])
 
-    step_bytes = algorithmic_bytes("fused", P, M)
+    step_bytes = algorithmic_bytes("fused", P, M, n_locals) + extra_streams * 4 * P
     l2_note = ("inputs per step exceed the 126 MB L2 many times over: no flush" if step_bytes > 8 * 126e6
                else "working set fits in L2: effective GB/s, not an HBM figure")
 
     for _ in range(max(3, args.warmup)):
-        ctx.fused_update(grads, 0, stream)
+        ctx.fused_update(grads, wid, stream)
     torch.cuda.synchronize()
     graph = None
     if args.graph:
@@ -213,7 +227,7 @@ def run_cuda(args):
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             for _ in range(args.graph):
-                ctx.fused_update(grads, 0)  # lands on the capturing stream
+                ctx.fused_update(grads, wid)  # lands on the capturing stream
         for _ in range(3):
             graph.replay()
         torch.cuda.synchronize()
@@ -225,7 +239,7 @@ def run_cuda(args):
         with ClockSampler(dev.index or 0) as clocks:
             ev[0].record(stream)
             for k in range(args.steps):
-                ctx.fused_update(grads, 0, stream)
+                ctx.fused_update(grads, wid, stream)
                 ev[k + 1].record(stream)
             torch.cuda.synchronize()
         gpu_launches = ctx.launch_count - launches_before
@@ -320,6 +334,7 @@ def run_cuda(args):
                    "n_params": P, "n_tensors": wl.n_tensors, "n_workers": M,
                    "bytes_per_step": step_bytes, "l2": l2_note,
                    "flavour": "deterministic" if args.deterministic else "default (FMA contraction allowed)",
+                   "variant": {"local_rule": args.local_rule, "locals_updated": n_locals, "multipliers": args.multipliers},
                    "launch": f"CUDA graph of {args.graph} steps, replayed" if args.graph else "one launch per step from the host",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),

@@ -50,6 +50,22 @@ namespace odsgd {
 constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
+#ifndef ODSGD_ALLDC_BATCH
+#define ODSGD_ALLDC_BATCH 1  // workers per batch when every worker's delay-compensated update is fused in
+#endif
+#ifndef ODSGD_ALLDC_UNROLL
+#define ODSGD_ALLDC_UNROLL 1  // vectors per thread in that case
+#endif
+#ifndef ODSGD_ALLSGD_BATCH
+#define ODSGD_ALLSGD_BATCH ODSGD_BATCH  // same, plain local rule for every worker
+#endif
+#ifndef ODSGD_ALLSGD_UNROLL
+#define ODSGD_ALLSGD_UNROLL ODSGD_UNROLL
+#endif
+constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
+constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
+constexpr int kAllSgdBatch = ODSGD_ALLSGD_BATCH;
+constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
 #if ODSGD_MIN_CTAS > 0
 #define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
 #else
@@ -251,23 +267,40 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
             v[u] = load_stream<NL>(a.v + off[u]);
         }
     }
+    // With every worker's delay-compensated local update in the pass, the previous local weights
+    // (and mean squares) are fetched in the same batch as the gradients, so a smaller batch
+    // keeps the register count in check.
+    constexpr bool kAllDc = LOCAL == kLocalAll && RULE != ODSGD_LOCAL_SGD;
+    constexpr int B = kAllDc ? kAllDcBatch : (LOCAL == kLocalAll ? kAllSgdBatch : kBatch);
     const int n_workers = a.n_workers;
-    for (int m0 = 0; m0 < n_workers; m0 += kBatch) {
-        Vec<NL> t[kBatch][U];
+    for (int m0 = 0; m0 < n_workers; m0 += B) {
+        Vec<NL> t[B][U], xv[B][U], msv[B][U];
         // independent loads first ...
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
+        for (int j = 0; j < B; ++j) {
             if (m0 + j < n_workers) {
                 const float* gp = a.g[m0 + j];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     if (ok[u]) t[j][u] = load_grad<NL>(gp + off[u]);
                 }
+                if (kAllDc) {
+                    float* xp = a.x[m0 + j];
+                    if (xp != nullptr) {
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            if (ok[u]) {
+                                xv[j][u] = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+                                if (RULE == ODSGD_LOCAL_DC_A) msv[j][u] = load_stream<NL>(a.ms[m0 + j] + off[u]);
+                            }
+                        }
+                    }
+                }
             }
         }
         // ... then the adds, strictly in worker order
 #pragma unroll
-        for (int j = 0; j < kBatch; ++j) {
+        for (int j = 0; j < B; ++j) {
             const int m = m0 + j;
             if (m < n_workers) {
 #pragma unroll
@@ -285,15 +318,14 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                         if (LOCAL == kLocalAll) {
                             float* xp = a.x[m];
                             if (xp != nullptr) {
-                                Vec<NL> xo, xv, msv;
-                                if (RULE != ODSGD_LOCAL_SGD) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
-                                if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[m] + off[u]);
+                                Vec<NL> xo;
 #pragma unroll
                                 for (int l = 0; l < NL; ++l) {
-                                    xo.e[l] = local_rule<DET, RULE>(w[u].e[l], t[j][u].e[l], xv.e[l], msv.e[l], a.lp);
+                                    xo.e[l] = local_rule<DET, RULE>(w[u].e[l], t[j][u].e[l], xv[j][u].e[l],
+                                                                    msv[j][u].e[l], a.lp);
                                 }
                                 store_stream<NL>(xp + off[u], xo);
-                                if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[m] + off[u], msv);
+                                if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[m] + off[u], msv[j][u]);
                             }
                         }
                     }
@@ -337,19 +369,22 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
     TensorCursor cur;
+    // vectors per thread: fewer when the pass also carries every worker's delay-compensated
+    // local update (three arenas per worker), where registers are the scarce resource
+    constexpr int UU = LOCAL != kLocalAll ? kUnroll : (RULE != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
     const unsigned long long nvec = a.n / NL;
-    const unsigned long long tile = (unsigned long long)blockDim.x * kUnroll;
+    const unsigned long long tile = (unsigned long long)blockDim.x * UU;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
     for (unsigned long long base = (unsigned long long)blockIdx.x * tile; base < nvec; base += stride) {
-        unsigned long long off[kUnroll];
-        bool ok[kUnroll];
+        unsigned long long off[UU];
+        bool ok[UU];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < UU; ++u) {
             const unsigned long long i = base + (unsigned long long)u * blockDim.x + threadIdx.x;
             ok[u] = i < nvec;
             off[u] = i * NL;
         }
-        server_vectors<DET, NL, LOCAL, RULE, MULT, kUnroll>(a, off, ok, cur);
+        server_vectors<DET, NL, LOCAL, RULE, MULT, UU>(a, off, ok, cur);
     }
     if (NL > 1) {
         // ragged tail: the last n % NL elements, one lane each
