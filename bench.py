@@ -79,6 +79,7 @@ def parse_args():
     ap.add_argument("--multipliers", action="store_true", help="per-tensor lr/wd multipliers (no decay off the weight tensors)")
     ap.add_argument("--local-rule", choices=["sgd", "dc_c", "dc_a"], default="sgd")
     ap.add_argument("--all-locals", action="store_true", help="update every worker's local weights in the fused pass")
+    ap.add_argument("--sweep-workers", default="", help="comma list of worker counts (<= the workload's) to time as well")
     ap.add_argument("--graph", type=int, default=0,
                     help="capture this many steps (even) in one CUDA graph and replay it; for the small, launch-bound sets")
     ap.add_argument("--no-e2e", action="store_true")
@@ -291,6 +292,31 @@ def run_cuda(args):
             b = algorithmic_bytes(name, P, M)
             extra[name] = {"ms": ms, "GBps": b / ms / 1e6, "frac": b / ms / 1e6 / peak}
 
+    # ---- worker-count sweep on the same arena (fused update, first m gradient buffers)
+    sweep = []
+    if args.sweep_workers and rank0:
+        for m in [int(x) for x in args.sweep_workers.split(",") if x]:
+            if m < 1 or m > M:
+                continue
+            loc = [local[0]] + [None] * (m - 1)
+            c2 = binding.Odsgd(w_a, v, n_workers=m, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                               w_b=w_b, local=loc, tensor_offsets=wl.offsets, flags=flags)
+            reps = max(20, min(200, args.steps))
+            for _ in range(3):
+                c2.fused_update(grads[:m], 0, stream)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                c2.fused_update(grads[:m], 0, stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            nb = algorithmic_bytes("fused", P, m)
+            sweep.append({"workers": m, "ms": ms, "GBps": nb / ms / 1e6, "frac": nb / ms / 1e6 / peak,
+                          "params_per_s": P / (ms * 1e-3), "bytes_per_step": nb})
+            c2.close()
+
     # ---- end to end: gradients start in pinned host memory, local weights come back
     e2e = None
     if not args.no_e2e:
@@ -349,6 +375,8 @@ def run_cuda(args):
         "step_ms": {"median": statistics.median(per_step), "min": min(per_step), "max": max(per_step)},
         "other_kernels": extra,
     }
+    if sweep:
+        line["worker_sweep"] = sweep
     print(json.dumps(line), flush=True)
     return 0
 

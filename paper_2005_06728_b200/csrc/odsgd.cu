@@ -159,19 +159,29 @@ int too_wide(odsgd_ctx* c, int block) {
     return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
 }
 
-template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
-int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
+int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
-    auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT>;
+    auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT, BB, UB>;
     static int cached_block = 0, cached_res = 0;
     if (cached_block != block) {
         cached_res = resident_ctas(kernel, block);
         cached_block = block;
     }
     if (cached_res == 0) return too_wide(c, block);
-    const int grid = grid_for(c, a.n, NL, block, kUnroll, kServerCtasPerSm);
+    const int grid = grid_for(c, a.n, NL, block, UB, kServerCtasPerSm);
     kernel<<<grid, block, 0, st>>>(a);
     return after_launch(c, "server kernel launch");
+}
+
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
+int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+    // few workers: the pass is close to a copy and wants the shallow, wide shape
+    if constexpr (LOCAL != kLocalAll) {
+        if (a.n_workers <= kFewWorkers)
+            return launch_server_k<DET, NL, LOCAL, RULE, MULT, kFewBatch, kFewUnroll>(c, a, st);
+    }
+    return launch_server_k<DET, NL, LOCAL, RULE, MULT, kBatch, kUnroll>(c, a, st);
 }
 
 template <bool DET, int NL, int LOCAL, int RULE>

@@ -47,8 +47,17 @@ namespace odsgd {
 #ifndef ODSGD_SMALL_UNROLL
 #define ODSGD_SMALL_UNROLL 4  // vectors per thread per tile in the local and ASGD kernels
 #endif
+#ifndef ODSGD_FEW_BATCH
+#define ODSGD_FEW_BATCH 2  // the same two knobs when there are at most kFewWorkers workers
+#endif
+#ifndef ODSGD_FEW_UNROLL
+#define ODSGD_FEW_UNROLL 4
+#endif
 constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
+constexpr int kFewBatch = ODSGD_FEW_BATCH;
+constexpr int kFewUnroll = ODSGD_FEW_UNROLL;
+constexpr int kFewWorkers = 4;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
 #ifndef ODSGD_ALLDC_BATCH
 #define ODSGD_ALLDC_BATCH 1  // workers per batch when every worker's delay-compensated update is fused in
@@ -255,7 +264,7 @@ __device__ __forceinline__ void find_tensor(const ServerArgs& a, unsigned long l
 // One vector (NL lanes) of the arena at element offset `off`:
 // sum the workers in order, apply the server rule, and (LOCAL != none) the
 // local rule for one worker or for every worker that has a local buffer.
-template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int U>
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int U>
 __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsigned long long (&off)[U],
                                                const bool (&ok)[U], TensorCursor& cur) {
     using O = Op<DET>;
@@ -271,7 +280,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
     // (and mean squares) are fetched in the same batch as the gradients, so a smaller batch
     // keeps the register count in check.
     constexpr bool kAllDc = LOCAL == kLocalAll && RULE != ODSGD_LOCAL_SGD;
-    constexpr int B = kAllDc ? kAllDcBatch : (LOCAL == kLocalAll ? kAllSgdBatch : kBatch);
+    constexpr int B = kAllDc ? kAllDcBatch : (LOCAL == kLocalAll ? kAllSgdBatch : BB);
     const int n_workers = a.n_workers;
     for (int m0 = 0; m0 < n_workers; m0 += B) {
         Vec<NL> t[B][U], xv[B][U], msv[B][U];
@@ -366,12 +375,15 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
     }
 }
 
-template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
+// BB x UB: gradient loads per batch x vectors per thread.  8 x 2 for many workers; with four
+// workers or fewer the kernel is close to a copy and 2 x 4 (fewer registers, more resident
+// warps, more vectors per thread) measured 7-20 % faster.
+template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
     TensorCursor cur;
     // vectors per thread: fewer when the pass also carries every worker's delay-compensated
     // local update (three arenas per worker), where registers are the scarce resource
-    constexpr int UU = LOCAL != kLocalAll ? kUnroll : (RULE != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
+    constexpr int UU = LOCAL != kLocalAll ? UB : (RULE != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * UU;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
@@ -384,7 +396,7 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
             ok[u] = i < nvec;
             off[u] = i * NL;
         }
-        server_vectors<DET, NL, LOCAL, RULE, MULT, UU>(a, off, ok, cur);
+        server_vectors<DET, NL, LOCAL, RULE, MULT, BB, UU>(a, off, ok, cur);
     }
     if (NL > 1) {
         // ragged tail: the last n % NL elements, one lane each
@@ -392,7 +404,7 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
         if (blockIdx.x == 0 && done + threadIdx.x < a.n) {
             const unsigned long long off1[1] = {done + threadIdx.x};
             const bool ok1[1] = {true};
-            server_vectors<DET, 1, LOCAL, RULE, MULT, 1>(a, off1, ok1, cur);
+            server_vectors<DET, 1, LOCAL, RULE, MULT, BB, 1>(a, off1, ok1, cur);
         }
     }
 }
