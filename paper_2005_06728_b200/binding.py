@@ -134,6 +134,24 @@ def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
     return s.cuda_stream
 
 
+class GradTable:
+    """The host array of device pointers the update calls take, built once from tensors that
+    stay alive (and are not reallocated) as long as the table is used."""
+
+    def __init__(self, grads: Sequence[torch.Tensor], n_workers: int, n_params: int):
+        if len(grads) != n_workers:
+            raise ValueError(f"need {n_workers} gradient tensors, got {len(grads)}")
+        self.tensors = list(grads)
+        self.n_workers, self.n_params = n_workers, n_params
+        self.table = _ptr_table([_dev_ptr(g, f"grads[{i}]", n_params) for i, g in enumerate(grads)])
+
+    def __len__(self) -> int:
+        return self.n_workers
+
+    def __iter__(self):
+        return iter(self.tensors)
+
+
 class Odsgd:
     """One context of the CUDA library (see include/odsgd.h for the semantics of each call)."""
 
@@ -183,10 +201,20 @@ class Odsgd:
         if rc != OK:
             raise OdsgdError(rc, self._lib.odsgd_last_error(self._h).decode())
 
-    def _grad_table(self, grads: Sequence[torch.Tensor]):
+    def _grad_table(self, grads):
+        if isinstance(grads, GradTable):
+            if grads.n_workers != self.n_workers or grads.n_params != self.n_params:
+                raise ValueError("gradient table was built for another context shape")
+            return grads.table
         if len(grads) != self.n_workers:
             raise ValueError(f"need {self.n_workers} gradient tensors, got {len(grads)}")
         return _ptr_table([_dev_ptr(g, f"grads[{i}]", self.n_params) for i, g in enumerate(grads)])
+
+    def grad_table(self, grads: Sequence[torch.Tensor]) -> "GradTable":
+        """Checks the gradient tensors once and keeps their pointer table, for loops that pass
+        the same buffers every iteration (saves the per-call marshalling, which dominates the
+        cost of a step on small parameter sets)."""
+        return GradTable(grads, self.n_workers, self.n_params)
 
     def close(self) -> None:
         if self._h:
@@ -202,7 +230,7 @@ class Odsgd:
     # -- the update calls
     def global_update(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
         self._check(self._lib.odsgd_global_update(self._h, self._grad_table(grads), _stream_handle(stream)))
-        self._bound = list(grads)
+        self._bound = grads
 
     def local_update(self, worker_id: int, stream: Optional[torch.cuda.Stream] = None) -> None:
         self._check(self._lib.odsgd_local_update(self._h, worker_id, _stream_handle(stream)))
@@ -211,7 +239,7 @@ class Odsgd:
                      stream: Optional[torch.cuda.Stream] = None) -> None:
         self._check(self._lib.odsgd_fused_update(self._h, self._grad_table(grads), worker_id,
                                                  _stream_handle(stream)))
-        self._bound = list(grads)
+        self._bound = grads
 
     def fused_update_host(self, host_grads: Sequence[torch.Tensor], dev_staging: Sequence[torch.Tensor],
                           worker_id: int, host_local_out: Optional[torch.Tensor] = None,
@@ -247,7 +275,7 @@ class Odsgd:
     def step_update(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
         """odsgd_step: one iteration of Algorithm 2's state machine (warm-up SSGD, then OD-SGD)."""
         self._check(self._lib.odsgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
-        self._bound = list(grads)
+        self._bound = grads
 
     def set_warmup(self, wp: int) -> None:
         self._check(self._lib.odsgd_set_warmup(self._h, wp))
@@ -286,7 +314,7 @@ class Odsgd:
 
         self._check(self._lib.odsgd_fused_update_mult_static(self._h, self._grad_table(grads), worker_id,
                                                              arr(lr_mult), arr(wd_mult), _stream_handle(stream)))
-        self._bound = list(grads)
+        self._bound = grads
 
     def set_server_mean_square(self, ms: Optional[torch.Tensor]) -> None:
         self._check(self._lib.odsgd_set_server_mean_square(self._h, _dev_ptr(ms, "mean_square", self.n_params)))

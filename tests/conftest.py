@@ -20,3 +20,12 @@ def cuda_device():
     if not torch.cuda.is_available():
         pytest.fail("a test marked gpu ran on a machine without a CUDA device")
     return torch.device("cuda:0")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_library():
+    """Compile libodsgd.so when it is missing or older than its sources (nvcc cross-compiles
+    without a GPU); a failed build fails the session loudly instead of skipping anything."""
+    from paper_2005_06728_b200 import build
+
+    return build.build()

@@ -507,3 +507,57 @@ def test_error_codes(cuda_device):
     ctx.fused_update(g, 0)
     torch.cuda.synchronize()
     assert ctx.launch_count == before + 1 and ctx.step == 2
+
+
+def test_prebuilt_gradient_table_gives_the_same_results(cuda_device):
+    wl = W.ragged_workload([30_000, 11], n_workers=4)
+    a, _, va, la = _ctx_for(wl, True, True)
+    b, _, vb, lb = _ctx_for(wl, True, True)
+    grads = W.make_grads(wl, 0, DEV)
+    table = a.grad_table(grads)
+    for _ in range(3):
+        a.fused_update(table, 0)
+        b.fused_update(grads, 0)
+    a.ssgd_step(table), b.ssgd_step(grads)
+    torch.cuda.synchronize()
+    assert torch.equal(a.weights(), b.weights()) and torch.equal(va, vb) and torch.equal(la[0], lb[0])
+    with pytest.raises(ValueError):
+        a.fused_update(binding.GradTable(grads[:2], 2, wl.arena_len), 0)  # built for two workers
+
+
+def test_arena_beyond_four_gibibytes_sampled(cuda_device):
+    """Element offsets past 2**32 bytes (and past 2**30 elements): 64-bit indexing everywhere.
+    One worker keeps the footprint at six arenas of 4.4 GB."""
+    n = (1 << 30) + (1 << 26) + 12_345 * 4 + 3  # > 2**30 elements, ragged tail of 3
+    free, _ = torch.cuda.mem_get_info()
+    if free < 7.5 * n * 4:
+        pytest.skip("needs about 33 GiB of device memory")
+    gen = torch.Generator(device=DEV).manual_seed(99)
+    w = torch.empty(n, device=DEV).normal_(0, 0.05, generator=gen)
+    v = torch.empty(n, device=DEV).normal_(0, 0.001, generator=gen)
+    g = torch.empty(n, device=DEV).normal_(0, 0.01, generator=gen)
+    w_b, x = torch.zeros(n, device=DEV), torch.zeros(n, device=DEV)
+    idx = np.unique(np.concatenate([np.arange(0, 4096), np.arange(n - 4096, n),
+                                    (1 << 30) + np.arange(-2048, 2048), (1 << 29) + np.arange(-64, 64),
+                                    np.random.default_rng(4).integers(0, n, 200_000)]))
+    idx_t = torch.from_numpy(idx).to(DEV)
+    hp = dict(lr=0.1, momentum=0.9, wd=1e-4)
+    ctx = binding.Odsgd(w, v, n_workers=1, local_lr=0.05, w_b=w_b, local=[x], flags=binding.FLAG_DETERMINISTIC, **hp)
+    w_ref, v_ref, g_s = w[idx_t].cpu().numpy(), v[idx_t].cpu().numpy(), g[idx_t].cpu().numpy()
+    ctx.fused_update([g], 0)
+    wp = np.empty_like(w_ref)
+    oracle.global_update([g_s], w_ref, v_ref, w_prev=wp, **hp)
+    torch.cuda.synchronize()
+    assert_bits(ctx.weights()[idx_t].cpu().numpy(), w_ref, "w")
+    assert_bits(v[idx_t].cpu().numpy(), v_ref, "v")
+    assert_bits(x[idx_t].cpu().numpy(), oracle.local_update(wp, g_s, local_lr=0.05), "x")
+    # the other kernels on the same arena: local update alone, ASGD step
+    x.zero_()
+    ctx.local_update(0)
+    ctx.asgd_step(0, g)
+    oracle.asgd_step(g_s, w_ref, v_ref, **hp)
+    torch.cuda.synchronize()
+    assert_bits(x[idx_t].cpu().numpy(), oracle.local_update(wp, g_s, local_lr=0.05), "x from the local kernel")
+    assert_bits(ctx.weights()[idx_t].cpu().numpy(), w_ref, "w after the ASGD step")
+    assert_bits(v[idx_t].cpu().numpy(), v_ref, "v after the ASGD step")
+    ctx.close()
