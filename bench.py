@@ -50,8 +50,7 @@ def measured_traffic(step_bytes):
 
     try:
         note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_alexnet_m8.md")).read()
-        src = b"".join(open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", f), "rb").read()
-                       for f in ("odsgd_kernels.cuh", "odsgd.cu"))
+        src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
         ratio = float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1))
         sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1)
     except (OSError, AttributeError, ValueError):

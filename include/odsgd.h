@@ -295,6 +295,17 @@ int odsgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream);
 int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights);
 
 /*
+ * Checkpoint / resume.  Every arena is the caller's, so saving them saves the state; what the
+ * context adds is the iteration index of the state machine above and the step counter.  To
+ * resume: create a context with the saved current global weights as w_a (plus v, the local
+ * arenas and, for ODSGD_LOCAL_DC_A, the mean-square arenas), choose the same rule and warm-up
+ * length, then restore the iteration index with odsgd_set_iteration (allowed at any time; it
+ * also lifts the "before the first odsgd_step" restriction of odsgd_set_warmup when set to 0).
+ */
+int odsgd_get_iteration(odsgd_ctx* ctx, uint64_t* iteration);
+int odsgd_set_iteration(odsgd_ctx* ctx, uint64_t iteration);
+
+/*
  * Learning-rate schedules the paper's runs use (Section 4): host-side helpers that return the
  * rate for iteration `step`; feed the result to odsgd_set_lr / odsgd_set_local_lr.
  *   step decay : base * factor^(number of boundaries <= step)       (divide by 10 at given epochs)

@@ -33,7 +33,7 @@ EXPORTS = (
     "odsgd_set_launch_config", "odsgd_get_launch_count", "odsgd_last_error",
     "odsgd_set_tensor_multipliers", "odsgd_dcasgd_step", "odsgd_set_server_mean_square", "odsgd_set_warmup",
     "odsgd_step", "odsgd_get_train_weights", "odsgd_lr_step_decay", "odsgd_lr_linear_ramp",
-    "odsgd_lr_poly_decay", "odsgd_fused_update_mult_static",
+    "odsgd_lr_poly_decay", "odsgd_fused_update_mult_static", "odsgd_get_iteration", "odsgd_set_iteration",
 )
 
 
@@ -101,6 +101,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_lr_step_decay": ([cf, cf, u64p, ctypes.c_size_t, ctypes.c_uint64], cf),
         "odsgd_lr_linear_ramp": ([cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
         "odsgd_lr_poly_decay": ([cf, cf, cf, ctypes.c_uint64, ctypes.c_uint64], cf),
+        "odsgd_get_iteration": ([vp, u64p], ci),
+        "odsgd_set_iteration": ([vp, ctypes.c_uint64], ci),
         "odsgd_fused_update_mult_static": ([vp, pvp, ci, ctypes.POINTER(cf), ctypes.POINTER(cf), vp], ci),
     }
     for name, (argtypes, restype) in sig.items():
@@ -368,6 +370,17 @@ class Odsgd:
     @step.setter
     def step(self, value: int) -> None:
         self._check(self._lib.odsgd_set_step(self._h, value))
+
+    @property
+    def iteration(self) -> int:
+        """Iteration index of the Algorithm 2 state machine (odsgd_step calls so far)."""
+        s = ctypes.c_uint64()
+        self._check(self._lib.odsgd_get_iteration(self._h, ctypes.byref(s)))
+        return s.value
+
+    @iteration.setter
+    def iteration(self, value: int) -> None:
+        self._check(self._lib.odsgd_set_iteration(self._h, value))
 
     @property
     def launch_count(self) -> int:

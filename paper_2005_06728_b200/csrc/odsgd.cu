@@ -53,12 +53,6 @@ namespace {
 
 thread_local std::string g_create_err;
 
-constexpr int kDefaultBlock = 256;       // server kernel
-constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels (measured best with 4 vectors per thread)
-// Grid cap of the kernels in CTAs per SM.  More CTAs than can be resident (two at this
-// register count) measured 1-2 % faster than an exactly persistent grid: late SMs pick up
-// the remaining tiles.
-constexpr int kServerCtasPerSm = 64;
 
 int fail(odsgd_ctx* ctx, int code, const std::string& msg) {
     if (ctx) ctx->err = msg; else g_create_err = msg;
@@ -754,6 +748,18 @@ int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights) {
     }
     if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
     *weights = c->local[worker_id];
+    return ODSGD_OK;
+}
+
+int odsgd_get_iteration(odsgd_ctx* ctx, uint64_t* iteration) {
+    if (!ctx || !iteration) return ODSGD_ERR_ARG;
+    *iteration = ctx->iter;
+    return ODSGD_OK;
+}
+
+int odsgd_set_iteration(odsgd_ctx* ctx, uint64_t iteration) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    ctx->iter = iteration;
     return ODSGD_OK;
 }
 

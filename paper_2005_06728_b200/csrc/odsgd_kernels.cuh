@@ -57,7 +57,10 @@ constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
 constexpr int kFewBatch = ODSGD_FEW_BATCH;
 constexpr int kFewUnroll = ODSGD_FEW_UNROLL;
-constexpr int kFewWorkers = 4;
+#ifndef ODSGD_FEW_WORKERS
+#define ODSGD_FEW_WORKERS 4
+#endif
+constexpr int kFewWorkers = ODSGD_FEW_WORKERS;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
 #ifndef ODSGD_ALLDC_BATCH
 #define ODSGD_ALLDC_BATCH 1  // workers per batch when every worker's delay-compensated update is fused in
@@ -80,6 +83,15 @@ constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
 #else
 #define ODSGD_SERVER_BOUNDS
 #endif
+
+// Launch shape (used by the host side; kept here so that everything that decides how the
+// kernels touch memory lives in one file).
+constexpr int kDefaultBlock = 256;       // server kernel
+constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels (measured best with 4 vectors per thread)
+// Grid cap of the kernels in CTAs per SM.  More CTAs than can be resident (two at the server
+// kernel's register count) measured 1-2 % faster than an exactly persistent grid: late SMs
+// pick up the remaining tiles.
+constexpr int kServerCtasPerSm = 64;
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
 

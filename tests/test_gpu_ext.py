@@ -253,3 +253,48 @@ def test_dcasgd_server_sequence(cuda_device, rule):
                 ms.copy_(torch.from_numpy(ms_ref))
         assert torch.all(v == 0), "Eq. 4/5 carry no momentum: v is untouched"
         ctx.close()
+
+
+def test_checkpoint_resume_reproduces_the_run(cuda_device):
+    """Stop after iteration 4 of a run with wp = 2 and the Eq. 5-6 local rule, rebuild a context
+    from the saved arenas and the saved iteration index, and finish: same bits as the
+    uninterrupted run."""
+    wl = W.ragged_workload([20_000, 9, 4_001], n_workers=2, lr=0.05, local_lr=0.04)
+    total, stop = 7, 4
+
+    def make(state=None):
+        if state is None:
+            w = W.make_weights(wl, DEV)
+            v = W.make_momentum(wl, DEV)
+            local = [torch.zeros_like(w) for _ in range(2)]
+            ms = [torch.zeros_like(w) for _ in range(2)]
+        else:
+            w, v, local, ms = state
+        ctx = binding.Odsgd(w, v, n_workers=2, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                            w_b=torch.zeros_like(w), local=local, tensor_offsets=wl.offsets,
+                            flags=binding.FLAG_DETERMINISTIC)
+        ctx.set_local_rule(binding.LOCAL_DC_A, 0.5, 0.9, 1e-6, ms)
+        ctx.set_warmup(2)
+        return ctx, v, local, ms
+
+    ref, v_ref, loc_ref, ms_ref = make()
+    for k in range(total):
+        ref.step_update(W.make_grads(wl, k, DEV))
+    a, v_a, loc_a, ms_a = make()
+    for k in range(stop):
+        a.step_update(W.make_grads(wl, k, DEV))
+    torch.cuda.synchronize()
+    saved = (a.weights().clone(), v_a.clone(), [t.clone() for t in loc_a], [t.clone() for t in ms_a])
+    saved_iter = a.iteration
+    assert saved_iter == stop
+    a.close()
+    b, v_b, loc_b, ms_b = make(saved)
+    b.iteration = saved_iter
+    for k in range(stop, total):
+        for m in range(2):
+            assert b.train_weights(m).data_ptr() == loc_b[m].data_ptr()
+        b.step_update(W.make_grads(wl, k, DEV))
+    torch.cuda.synchronize()
+    assert torch.equal(b.weights(), ref.weights()) and torch.equal(v_b, v_ref)
+    for m in range(2):
+        assert torch.equal(loc_b[m], loc_ref[m]) and torch.equal(ms_b[m], ms_ref[m])
