@@ -8,7 +8,8 @@
 //   * the M gradient streams are fetched in batches of kBatch x kUnroll
 //     independent 128-bit loads per thread before the dependent adds start
 //     (about 160 KB in flight per SM at two resident CTAs); the adds themselves
-//     stay in worker order 0..M-1;
+//     stay in worker order 0..M-1; with few workers, or with every worker's
+//     local update fused in, shallower batches and more resident warps win;
 //   * gradients go through the read-only path (ld.global.nc), which measured
 //     5-8 % faster here than streaming loads (ld.global.cs); state that is read
 //     and written by the same kernel uses coherent loads; results are stored
@@ -26,58 +27,69 @@
 
 namespace odsgd {
 
+// ------------------------------------------------------------------ tuning constants
+// Each can be overridden with -D for a sweep; the defaults are what measured best on B200.
+
+// Server kernel, general case: gradient loads per batch x vectors per thread.
 #ifndef ODSGD_BATCH
-#define ODSGD_BATCH 8  // gradient loads in flight per thread and vector
+#define ODSGD_BATCH 8
 #endif
 #ifndef ODSGD_UNROLL
-#define ODSGD_UNROLL 2  // vectors per thread per tile
+#define ODSGD_UNROLL 2
 #endif
-#ifndef ODSGD_GRAD_LOAD
-#define ODSGD_GRAD_LOAD 1  // 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching
-#endif
-#ifndef ODSGD_STORE
-#define ODSGD_STORE 0  // 0 streaming (st.global.cs), 1 default caching
-#endif
-#ifndef ODSGD_MIN_CTAS
-#define ODSGD_MIN_CTAS 0  // > 0: __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS) on the server kernel
-#endif
-#ifndef ODSGD_MAX_BLOCK
-#define ODSGD_MAX_BLOCK 256
-#endif
-#ifndef ODSGD_SMALL_UNROLL
-#define ODSGD_SMALL_UNROLL 4  // vectors per thread per tile in the local and ASGD kernels
+// Server kernel with at most ODSGD_FEW_WORKERS workers (the pass is close to a 1:1 copy).
+#ifndef ODSGD_FEW_WORKERS
+#define ODSGD_FEW_WORKERS 4
 #endif
 #ifndef ODSGD_FEW_BATCH
-#define ODSGD_FEW_BATCH 2  // the same two knobs when there are at most kFewWorkers workers
+#define ODSGD_FEW_BATCH 2
 #endif
 #ifndef ODSGD_FEW_UNROLL
 #define ODSGD_FEW_UNROLL 4
 #endif
-constexpr int kBatch = ODSGD_BATCH;
-constexpr int kUnroll = ODSGD_UNROLL;
-constexpr int kFewBatch = ODSGD_FEW_BATCH;
-constexpr int kFewUnroll = ODSGD_FEW_UNROLL;
-#ifndef ODSGD_FEW_WORKERS
-#define ODSGD_FEW_WORKERS 4
-#endif
-constexpr int kFewWorkers = ODSGD_FEW_WORKERS;
-constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
-#ifndef ODSGD_ALLDC_BATCH
-#define ODSGD_ALLDC_BATCH 1  // workers per batch when every worker's delay-compensated update is fused in
-#endif
-#ifndef ODSGD_ALLDC_UNROLL
-#define ODSGD_ALLDC_UNROLL 1  // vectors per thread in that case
-#endif
+// Server kernel with every worker's local update in the pass: plain rule / Eq. 4, Eq. 5-6.
 #ifndef ODSGD_ALLSGD_BATCH
-#define ODSGD_ALLSGD_BATCH ODSGD_BATCH  // same, plain local rule for every worker
+#define ODSGD_ALLSGD_BATCH ODSGD_BATCH
 #endif
 #ifndef ODSGD_ALLSGD_UNROLL
 #define ODSGD_ALLSGD_UNROLL ODSGD_UNROLL
 #endif
-constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
-constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
+#ifndef ODSGD_ALLDC_BATCH
+#define ODSGD_ALLDC_BATCH 1
+#endif
+#ifndef ODSGD_ALLDC_UNROLL
+#define ODSGD_ALLDC_UNROLL 1
+#endif
+// Local and ASGD kernels: vectors per thread per tile.
+#ifndef ODSGD_SMALL_UNROLL
+#define ODSGD_SMALL_UNROLL 4
+#endif
+// Gradient loads: 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching.
+#ifndef ODSGD_GRAD_LOAD
+#define ODSGD_GRAD_LOAD 1
+#endif
+// Stores: 0 streaming (st.global.cs), 1 default caching.
+#ifndef ODSGD_STORE
+#define ODSGD_STORE 0
+#endif
+// > 0: __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS) on the server kernel (register cap).
+#ifndef ODSGD_MIN_CTAS
+#define ODSGD_MIN_CTAS 0
+#endif
+#ifndef ODSGD_MAX_BLOCK
+#define ODSGD_MAX_BLOCK 256
+#endif
+
+constexpr int kBatch = ODSGD_BATCH;
+constexpr int kUnroll = ODSGD_UNROLL;
+constexpr int kFewWorkers = ODSGD_FEW_WORKERS;
+constexpr int kFewBatch = ODSGD_FEW_BATCH;
+constexpr int kFewUnroll = ODSGD_FEW_UNROLL;
 constexpr int kAllSgdBatch = ODSGD_ALLSGD_BATCH;
 constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
+constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
+constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
+constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
 #if ODSGD_MIN_CTAS > 0
 #define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
 #else
@@ -87,10 +99,10 @@ constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
 // Launch shape (used by the host side; kept here so that everything that decides how the
 // kernels touch memory lives in one file).
 constexpr int kDefaultBlock = 256;       // server kernel
-constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels (measured best with 4 vectors per thread)
-// Grid cap of the kernels in CTAs per SM.  More CTAs than can be resident (two at the server
-// kernel's register count) measured 1-2 % faster than an exactly persistent grid: late SMs
-// pick up the remaining tiles.
+constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels
+// Grid cap in CTAs per SM.  More CTAs than can be resident (two at the server kernel's
+// register count) measured 1-2 % faster than an exactly persistent grid: late SMs pick up
+// the remaining tiles.
 constexpr int kServerCtasPerSm = 64;
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
