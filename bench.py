@@ -390,7 +390,16 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
-    return run_cuda(args)
+    try:
+        return run_cuda(args)
+    finally:
+        try:
+            import torch.distributed as dist
+
+            if dist.is_available() and dist.is_initialized():
+                dist.destroy_process_group()
+        except Exception:
+            pass
 
 
 if __name__ == "__main__":
