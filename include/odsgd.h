@@ -167,11 +167,17 @@ int odsgd_fused_update(odsgd_ctx* ctx, const float* const* worker_grads, int wor
  * pointers (page-locked memory for real asynchrony), n_params floats each.
  * `dev_staging`: host array of n_workers device pointers the gradients are copied
  * into (caller-owned, n_params floats each).  If `host_local_out` is not NULL and
- * worker_id >= 0, local[worker_id] is copied back to it after the update.  All copies
- * and the kernel are enqueued on `stream` in order; nothing is synchronised.
+ * worker_id >= 0, local[worker_id] is copied back to it after the update.  The uploads and
+ * the kernel are enqueued on `stream` in order; nothing is synchronised.
+ * `copy_stream`: NULL (or equal to `stream`) puts the copy-back on `stream` too.  A different
+ * stream makes the copy-back run there, ordered after the kernel by an event, so that it
+ * overlaps the NEXT call's uploads (the bus is full duplex); the next call's kernel waits for
+ * that copy before it overwrites local[worker_id].  The caller synchronises `copy_stream`
+ * before reading `host_local_out`.  (The context creates two CUDA events on first use of a
+ * separate copy stream.)
  */
 int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging,
-                            int worker_id, float* host_local_out, void* stream);
+                            int worker_id, float* host_local_out, void* stream, void* copy_stream);
 
 /*
  * SSGD server step (Section 3.1): the same arithmetic as the global update, applied

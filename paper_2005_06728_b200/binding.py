@@ -78,7 +78,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_global_update": ([vp, pvp, vp], ci),
         "odsgd_local_update": ([vp, ci, vp], ci),
         "odsgd_fused_update": ([vp, pvp, ci, vp], ci),
-        "odsgd_fused_update_host": ([vp, pvp, pvp, ci, vp, vp], ci),
+        "odsgd_fused_update_host": ([vp, pvp, pvp, ci, vp, vp, vp], ci),
         "odsgd_ssgd_step": ([vp, pvp, vp], ci),
         "odsgd_asgd_step": ([vp, ci, vp, vp], ci),
         "odsgd_set_lr": ([vp, cf], ci),
@@ -245,7 +245,8 @@ class Odsgd:
 
     def fused_update_host(self, host_grads: Sequence[torch.Tensor], dev_staging: Sequence[torch.Tensor],
                           worker_id: int, host_local_out: Optional[torch.Tensor] = None,
-                          stream: Optional[torch.cuda.Stream] = None) -> None:
+                          stream: Optional[torch.cuda.Stream] = None,
+                          copy_stream: Optional[torch.cuda.Stream] = None) -> None:
         if len(host_grads) != self.n_workers:
             raise ValueError(f"need {self.n_workers} host gradient tensors")
         hp = []
@@ -260,7 +261,8 @@ class Odsgd:
                 raise TypeError("host_local_out: need a contiguous float32 CPU tensor of n_params elements")
             out_ptr = t.data_ptr()
         self._check(self._lib.odsgd_fused_update_host(self._h, _ptr_table(hp), self._grad_table(dev_staging),
-                                                      worker_id, out_ptr, _stream_handle(stream)))
+                                                      worker_id, out_ptr, _stream_handle(stream),
+                                                      copy_stream.cuda_stream if copy_stream is not None else None))
         self._bound = list(dev_staging)
 
     def ssgd_step(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
@@ -415,8 +417,8 @@ def odsgd_fused_update(ctx: Odsgd, worker_grads, worker_id: int, stream=None) ->
 
 
 def odsgd_fused_update_host(ctx: Odsgd, host_grads, dev_staging, worker_id: int, host_local_out=None,
-                            stream=None) -> None:
-    ctx.fused_update_host(host_grads, dev_staging, worker_id, host_local_out, stream)
+                            stream=None, copy_stream=None) -> None:
+    ctx.fused_update_host(host_grads, dev_staging, worker_id, host_local_out, stream, copy_stream)
 
 
 def odsgd_ssgd_step(ctx: Odsgd, worker_grads, stream=None) -> None:

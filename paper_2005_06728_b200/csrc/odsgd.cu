@@ -46,6 +46,10 @@ struct odsgd_ctx {
     float* server_ms = nullptr;  // Eq. 6 state of the server-side DC-ASGD step
     uint64_t wp = 0;             // Algorithm 2's warm-up length
     uint64_t iter = 0;           // iterations done through odsgd_step
+    // host-buffer entry point with a separate copy stream: ordering between the two streams
+    cudaEvent_t ev_kernel_done = nullptr;  // recorded on the compute stream after the update kernel
+    cudaEvent_t ev_copy_done = nullptr;    // recorded on the copy stream after the device-to-host copy
+    bool copy_pending = false;
     std::string err;
 };
 
@@ -273,6 +277,16 @@ LocalParams local_params(const odsgd_ctx* c) {
     return p;
 }
 
+// A copy-back of local weights that odsgd_fused_update_host put on a separate copy stream
+// must be out before any later kernel overwrites a local arena: make `st` wait for it.
+int settle_copy(odsgd_ctx* c, cudaStream_t st) {
+    if (!c->copy_pending) return ODSGD_OK;
+    const cudaError_t e = cudaStreamWaitEvent(st, c->ev_copy_done, 0);
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("stream wait: ") + cudaGetErrorString(e));
+    c->copy_pending = false;
+    return ODSGD_OK;
+}
+
 // Checks a table of gradient pointers against the context's state buffers.
 int check_grads(odsgd_ctx* c, const float* const* grads, std::vector<Named>* ptrs) {
     if (!grads) return fail(c, ODSGD_ERR_ARG, "worker_grads is NULL");
@@ -382,6 +396,8 @@ int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
             if (o % 4 != 0) { lanes = 1; break; }
     }
 
+    rc = settle_copy(c, static_cast<cudaStream_t>(stream));
+    if (rc != ODSGD_OK) return rc;
     rc = launch_server(c, a, lanes, local_mode, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
 
@@ -478,6 +494,8 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
 int odsgd_destroy(odsgd_ctx* ctx) {
     if (!ctx) return ODSGD_ERR_ARG;
     if (ctx->table_dev) cudaFree(ctx->table_dev);
+    if (ctx->ev_kernel_done) cudaEventDestroy(ctx->ev_kernel_done);
+    if (ctx->ev_copy_done) cudaEventDestroy(ctx->ev_copy_done);
     delete ctx;
     return ODSGD_OK;
 }
@@ -517,11 +535,13 @@ int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     if (need_ms) ptrs.push_back({a.ms, "mean_square", worker_id});
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
+    const int rc_copy = settle_copy(c, static_cast<cudaStream_t>(stream));
+    if (rc_copy != ODSGD_OK) return rc_copy;
     return launch_local(c, a, lanes, false, static_cast<cudaStream_t>(stream));
 }
 
 int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging, int worker_id,
-                            float* host_local_out, void* stream) {
+                            float* host_local_out, void* stream, void* copy_stream) {
     if (!ctx) return ODSGD_ERR_ARG;
     odsgd_ctx* c = ctx;
     if (!host_grads || !dev_staging) return fail(c, ODSGD_ERR_ARG, "host_grads / dev_staging is NULL");
@@ -539,10 +559,28 @@ int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, floa
         const cudaError_t e = cudaMemcpyAsync(dev_staging[m], host_grads[m], bytes, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("host-to-device copy: ") + cudaGetErrorString(e));
     }
+    cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
+    const bool split = host_local_out && copy_stream && cs != st;
+    if (split && (!c->ev_kernel_done || !c->ev_copy_done)) {
+        cudaError_t e = cudaSuccess;
+        if (!c->ev_kernel_done) e = cudaEventCreateWithFlags(&c->ev_kernel_done, cudaEventDisableTiming);
+        if (e == cudaSuccess && !c->ev_copy_done) e = cudaEventCreateWithFlags(&c->ev_copy_done, cudaEventDisableTiming);
+        if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("event creation: ") + cudaGetErrorString(e));
+    }
     rc = server_call(c, dev_staging, true, worker_id, stream);
     if (rc != ODSGD_OK) return rc;
     if (host_local_out) {
-        const cudaError_t e = cudaMemcpyAsync(host_local_out, c->local[worker_id], bytes, cudaMemcpyDeviceToHost, st);
+        cudaError_t e = cudaSuccess;
+        if (split) {
+            e = cudaEventRecord(c->ev_kernel_done, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, c->ev_kernel_done, 0);
+        }
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(host_local_out, c->local[worker_id], bytes, cudaMemcpyDeviceToHost, split ? cs : st);
+        if (e == cudaSuccess && split) {
+            e = cudaEventRecord(c->ev_copy_done, cs);
+            c->copy_pending = e == cudaSuccess;
+        }
         if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("device-to-host copy: ") + cudaGetErrorString(e));
     }
     return ODSGD_OK;
@@ -708,6 +746,8 @@ int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* st
     if (need_ms) ptrs.push_back({a.ms, "server_mean_square", -1});
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
+    const int rc_copy = settle_copy(c, static_cast<cudaStream_t>(stream));
+    if (rc_copy != ODSGD_OK) return rc_copy;
     const int rc = launch_local(c, a, lanes, true, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
     c->step += 1;
@@ -942,6 +982,8 @@ int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_gr
     a.t_wd_mult = a.t_lr_mult + nt;
     a.n_tensors = (unsigned int)nt;
 
+    rc = settle_copy(c, st);
+    if (rc != ODSGD_OK) return rc;
     const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
     if (det)
         rc = lanes == 4 ? launch_server_m<true, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)

@@ -118,7 +118,7 @@ def test_null_context_is_an_argument_error(lib):
     assert lib.odsgd_global_update(null, None, None) == binding.ERR_ARG
     assert lib.odsgd_local_update(null, 0, None) == binding.ERR_ARG
     assert lib.odsgd_fused_update(null, None, 0, None) == binding.ERR_ARG
-    assert lib.odsgd_fused_update_host(null, None, None, 0, None, None) == binding.ERR_ARG
+    assert lib.odsgd_fused_update_host(null, None, None, 0, None, None, None) == binding.ERR_ARG
     assert lib.odsgd_ssgd_step(null, None, None) == binding.ERR_ARG
     assert lib.odsgd_asgd_step(null, 0, None, None) == binding.ERR_ARG
     assert lib.odsgd_set_lr(null, 0.1) == binding.ERR_ARG

@@ -297,6 +297,34 @@ def test_host_buffer_entry_point(cuda_device):
         torch.cuda.synchronize()
         assert torch.equal(ctx.weights(), ref.weights())
         assert torch.equal(out, lr_[1].cpu()) and torch.equal(local[1], lr_[1])
+    # copy-back on a stream of its own, overlapping the next call's uploads: same results, and a
+    # plain update issued right after still waits for the copy before touching the local arena
+    side = torch.cuda.Stream()
+    outs = []
+    for it in range(2, 5):
+        hg = [W.make_grad(wl, m, it).pin_memory() for m in range(3)]
+        o = torch.empty(wl.arena_len, dtype=torch.float32).pin_memory()
+        ctx.fused_update_host(hg, staging, 1, o, None, side)
+        ref.fused_update([g.to(DEV) for g in hg], 1)
+        torch.cuda.synchronize()
+        outs.append((o, lr_[1].cpu()))
+    for o, want in outs:
+        assert torch.equal(o, want)
+    hg = [W.make_grad(wl, m, 9).pin_memory() for m in range(3)]
+    o = torch.empty(wl.arena_len, dtype=torch.float32).pin_memory()
+    ctx.fused_update_host(hg, staging, 1, o, None, side)
+    ref.fused_update([g.to(DEV) for g in hg], 1)
+    torch.cuda.synchronize()
+    want = lr_[1].cpu()
+    g2 = W.make_grads(wl, 10, DEV)
+    ctx.fused_update_host(hg, staging, 1, o, None, side)   # copy-back in flight on `side` ...
+    ctx.fused_update(g2, 1)                                # ... when the next kernel rewrites local[1]
+    ref.fused_update([g.to(DEV) for g in hg], 1)
+    ref_after_first = lr_[1].clone()
+    ref.fused_update(g2, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(o, ref_after_first.cpu()), "the copy saw the weights of its own step"
+    assert torch.equal(local[1], lr_[1]) and torch.equal(ctx.weights(), ref.weights())
 
 
 def test_cuda_graph_replay_matches_eager_calls(cuda_device):
