@@ -116,6 +116,12 @@ def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
 
     cut, w, v, grads = oracle_sample(wl, n_workers, sample_elems)
     s = w.size
+    old_affinity = None
+    try:  # one core, as the oracle is single-threaded; keeps the figure free of migrations
+        old_affinity = os.sched_getaffinity(0)
+        os.sched_setaffinity(0, {sorted(old_affinity)[-1]})
+    except (AttributeError, OSError):
+        old_affinity = None
     wp = np.empty_like(w)
     x = np.empty_like(w)
     times = []
@@ -129,7 +135,12 @@ def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
             times.append(dt)
         if it >= warmup + 2 and time.perf_counter() - t_start > budget_s:
             break
-    sec = statistics.mean(times)
+    if old_affinity:
+        try:
+            os.sched_setaffinity(0, old_affinity)
+        except OSError:
+            pass
+    sec = statistics.median(times)
     nbytes = algorithmic_bytes("fused", s, n_workers)
     info = {"value": nbytes / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
             "sample": f"first {s} of {wl.arena_len} elements of {wl.name}, all {n_workers} workers, "
