@@ -72,7 +72,8 @@ def parse_args():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default="vgg16", help="lenet5 | resnet56 | alexnet | resnet50 | vgg16")
     ap.add_argument("--workers", type=int, default=0, help="override the workload's worker count")
-    ap.add_argument("--deterministic", action="store_true", help="time the one-rounding-per-operator flavour")
+    ap.add_argument("--allow-fma", action="store_true",
+                    help="time the flavour in which multiply-add pairs may fuse (default: one rounding per operator)")
     ap.add_argument("--block", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--multipliers", action="store_true", help="per-tensor lr/wd multipliers (no decay off the weight tensors)")
@@ -213,7 +214,7 @@ def run_cuda(args):
     local = [w_a.clone() for _ in range(n_locals)] + [None] * (M - n_locals)
     sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
     grads = [W.make_grad(wl, m, 0, dev, _sigma=sg, _pads=pads) for m in range(M)]
-    flags = binding.FLAG_DETERMINISTIC if args.deterministic else 0
+    flags = binding.FLAG_ALLOW_FMA if args.allow_fma else 0
     ctx = binding.Odsgd(w_a, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
                         w_b=w_b, local=local, tensor_offsets=wl.offsets, flags=flags)
     if args.block or args.ctas_per_sm:
@@ -378,7 +379,7 @@ def run_cuda(args):
         "config": {"workload": workload_label(wl, M),
                    "n_params": P, "n_tensors": wl.n_tensors, "n_workers": M,
                    "bytes_per_step": step_bytes, "l2": l2_note,
-                   "flavour": "deterministic" if args.deterministic else "default (FMA contraction allowed)",
+                   "flavour": "FMA contraction allowed" if args.allow_fma else "default: one rounding per operator, bit-exact against the CPU oracle",
                    "variant": {"local_rule": args.local_rule, "locals_updated": n_locals, "multipliers": args.multipliers},
                    "launch": f"CUDA graph of {args.graph} steps, replayed" if args.graph else "one launch per step from the host",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},

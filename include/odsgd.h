@@ -40,10 +40,11 @@
  *     ODSGD_FLAG_ALLOW_UNALIGNED a misaligned pointer is rejected with ODSGD_ERR_ALIGN;
  *     with it, a scalar (4-byte) kernel is used for that call.
  *   - Arithmetic is IEEE-754 binary32, round-to-nearest-even, subnormals kept.  By
- *     default the compiler may fuse a multiply with the following add (one rounding
- *     instead of two).  With ODSGD_FLAG_DETERMINISTIC every operator written above
- *     rounds on its own, so results are reproducible bit for bit against a plain
- *     scalar CPU evaluation in the same order.
+ *     default every operator written above rounds on its own, so results are
+ *     reproducible bit for bit against a plain scalar CPU evaluation in the same order
+ *     (the kernels are bound by memory bandwidth, so this costs no time).  With
+ *     ODSGD_FLAG_ALLOW_FMA the compiler may fuse a multiply with the following add (one
+ *     rounding instead of two); results then differ from the default in the last bits.
  */
 #ifndef ODSGD_H_
 #define ODSGD_H_
@@ -69,8 +70,9 @@ extern "C" {
 #define ODSGD_ERR_CUDA (-5)        /* a CUDA runtime call or the launch failed; text in odsgd_last_error */
 #define ODSGD_ERR_UNSUPPORTED (-6) /* valid request this build does not implement */
 
-#define ODSGD_FLAG_DETERMINISTIC 0x1u   /* no fused multiply-add: one rounding per operator */
+#define ODSGD_FLAG_DETERMINISTIC 0x1u   /* one rounding per operator; this is the default, the bit only states it */
 #define ODSGD_FLAG_ALLOW_UNALIGNED 0x2u /* accept 4-byte aligned pointers (slower scalar kernel) */
+#define ODSGD_FLAG_ALLOW_FMA 0x4u       /* let multiply-add pairs fuse (excludes ODSGD_FLAG_DETERMINISTIC) */
 
 /* Local update rules (Section 3.3, "Local Updater"). */
 #define ODSGD_LOCAL_SGD 0  /* x = w_bak - local_lr * g */

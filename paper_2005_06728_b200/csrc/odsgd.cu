@@ -208,7 +208,7 @@ int launch_server_l(odsgd_ctx* c, const ServerArgs& a, int local_mode, cudaStrea
 }
 
 int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, cudaStream_t st) {
-    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
     if (det) return lanes == 4 ? launch_server_l<true, 4>(c, a, local_mode, st) : launch_server_l<true, 1>(c, a, local_mode, st);
     return lanes == 4 ? launch_server_l<false, 4>(c, a, local_mode, st) : launch_server_l<false, 1>(c, a, local_mode, st);
 }
@@ -241,7 +241,7 @@ int launch_local_r(odsgd_ctx* c, const LocalArgs& a, bool server, cudaStream_t s
 }
 
 int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, bool server, cudaStream_t st) {
-    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
     if (det) return lanes == 4 ? launch_local_r<true, 4>(c, a, server, st) : launch_local_r<true, 1>(c, a, server, st);
     return lanes == 4 ? launch_local_r<false, 4>(c, a, server, st) : launch_local_r<false, 1>(c, a, server, st);
 }
@@ -261,7 +261,7 @@ int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
 }
 
 int launch_asgd(odsgd_ctx* c, const AsgdArgs& a, int lanes, cudaStream_t st) {
-    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
     if (det) return lanes == 4 ? launch_asgd_t<true, 4>(c, a, st) : launch_asgd_t<true, 1>(c, a, st);
     return lanes == 4 ? launch_asgd_t<false, 4>(c, a, st) : launch_asgd_t<false, 1>(c, a, st);
 }
@@ -444,8 +444,10 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
     for (size_t t = 0; t < d->n_tensors; ++t)
         if (d->tensor_offsets[t + 1] <= d->tensor_offsets[t])
             return fail(nullptr, ODSGD_ERR_ARG, "tensor_offsets must be strictly ascending (at tensor " + std::to_string(t) + ")");
-    if (d->flags & ~(ODSGD_FLAG_DETERMINISTIC | ODSGD_FLAG_ALLOW_UNALIGNED))
+    if (d->flags & ~(ODSGD_FLAG_DETERMINISTIC | ODSGD_FLAG_ALLOW_UNALIGNED | ODSGD_FLAG_ALLOW_FMA))
         return fail(nullptr, ODSGD_ERR_ARG, "unknown flag bits");
+    if ((d->flags & ODSGD_FLAG_DETERMINISTIC) && (d->flags & ODSGD_FLAG_ALLOW_FMA))
+        return fail(nullptr, ODSGD_ERR_ARG, "ODSGD_FLAG_DETERMINISTIC and ODSGD_FLAG_ALLOW_FMA exclude each other");
 
     odsgd_ctx* c = new (std::nothrow) odsgd_ctx;
     if (!c) return fail(nullptr, ODSGD_ERR_ARG, "out of host memory");
@@ -984,7 +986,7 @@ int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_gr
 
     rc = settle_copy(c, st);
     if (rc != ODSGD_OK) return rc;
-    const bool det = (c->flags & ODSGD_FLAG_DETERMINISTIC) != 0;
+    const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
     if (det)
         rc = lanes == 4 ? launch_server_m<true, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)
                         : launch_server_m<true, 1, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st);

@@ -51,7 +51,7 @@ class GpuImpl(Impl):
     """The CUDA library driven through its C ABI, one fresh context per call."""
 
     def __init__(self, deterministic: bool = True, pingpong: bool = True, fused: bool = False):
-        self.flags = binding.FLAG_DETERMINISTIC if deterministic else 0
+        self.flags = binding.FLAG_DETERMINISTIC if deterministic else binding.FLAG_ALLOW_FMA
         self.pingpong = pingpong
         self.fused = fused
 

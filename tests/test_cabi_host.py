@@ -67,6 +67,7 @@ def _create(lib, d):
     (dict(w_b=0x30000, w_delayed=0x40000), binding.ERR_ARG, "w_delayed"),
     (dict(n_tensors=0), binding.ERR_ARG, "tensor_offsets"),
     (dict(flags=0x80), binding.ERR_ARG, "flag"),
+    (dict(flags=binding.FLAG_DETERMINISTIC | binding.FLAG_ALLOW_FMA), binding.ERR_ARG, "exclude"),
     (dict(w_a=0x10004), binding.ERR_ALIGN, "w_a"),
     (dict(v=0x10000 + 4 * 1000), binding.ERR_OVERLAP, "overlaps"),
     (dict(w_b=0x20000 + 16), binding.ERR_OVERLAP, "overlaps"),

@@ -50,7 +50,7 @@ def test_multipliers_on_many_small_tensors(cuda_device, name):
         local = [torch.zeros_like(w) for _ in range(M)]
         ctx = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
                             w_b=torch.zeros_like(w), local=local, tensor_offsets=wl.offsets,
-                            flags=binding.FLAG_DETERMINISTIC if det else 0)
+                            flags=binding.FLAG_DETERMINISTIC if det else binding.FLAG_ALLOW_FMA)
         ctx.set_tensor_multipliers(lr_mult.tolist(), wd_mult.tolist())
         w_ref, v_ref = w.cpu().numpy().copy(), v.cpu().numpy().copy()
         for it in range(4):
@@ -217,7 +217,7 @@ def test_dcasgd_server_sequence(cuda_device, rule):
         local = [w.clone() for _ in range(3)]
         ms = torch.zeros_like(w)
         ctx = binding.Odsgd(w, v, n_workers=3, lr=wl.lr, local_lr=9.0, momentum=0.9, wd=0.5, local=local,
-                            flags=binding.FLAG_DETERMINISTIC if det else 0)
+                            flags=binding.FLAG_DETERMINISTIC if det else binding.FLAG_ALLOW_FMA)
         with pytest.raises(binding.OdsgdError) as e:
             ctx.dcasgd_step(0, W.make_grad(wl, 0, 0, DEV))
         assert e.value.code == binding.ERR_STATE  # rule still SGD

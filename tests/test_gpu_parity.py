@@ -59,7 +59,7 @@ def _run_fused(w, v, grads, *, det, pingpong, worker_id, hp, launch=None, unalig
     """One fused call on fresh buffers; returns dict of numpy results."""
     n, nw = w.size, len(grads)
     lr, llr, mu, wd = hp
-    flags = (binding.FLAG_DETERMINISTIC if det else 0) | (binding.FLAG_ALLOW_UNALIGNED if unaligned else 0)
+    flags = (binding.FLAG_DETERMINISTIC if det else binding.FLAG_ALLOW_FMA) | (binding.FLAG_ALLOW_UNALIGNED if unaligned else 0)
     bufs = []
 
     def put(x):
@@ -161,6 +161,22 @@ def test_default_build_within_tolerance(cuda_device, n):
         assert_bits(r["w_prev"], wp, "backup is a copy")
 
 
+def test_plain_flags_are_the_exact_flavour(cuda_device):
+    """flags = 0 already rounds every operator on its own: bit-exact against the oracle, and the
+    same bits as with ODSGD_FLAG_DETERMINISTIC spelled out."""
+    n, nw = 50_003, 5
+    w, v, grads = _case(n, nw, seed=77)
+    wo, vo, wp, xs = _oracle_fused(w, v, grads, HP)
+    wa, va, oth, x = (torch.from_numpy(a).to(DEV) for a in (w, v, np.zeros(n, np.float32), np.zeros(n, np.float32)))
+    ctx = binding.Odsgd(wa, va, n_workers=nw, lr=HP[0], local_lr=HP[1], momentum=HP[2], wd=HP[3], w_b=oth,
+                        local=[None] * (nw - 1) + [x])
+    ctx.fused_update([torch.from_numpy(g).to(DEV) for g in grads], nw - 1)
+    torch.cuda.synchronize()
+    assert_bits(ctx.weights().cpu().numpy(), wo, "w")
+    assert_bits(va.cpu().numpy(), vo, "v")
+    assert_bits(x.cpu().numpy(), xs[nw - 1], "x")
+
+
 @pytest.mark.parametrize("launch", [(64, 1), (128, 3), (512, 0), (96, 2), (256, 16)])
 def test_launch_shapes_do_not_change_results(cuda_device, launch):
     n, nw = 200_003, 6
@@ -213,7 +229,7 @@ def _ctx_for(wl, det, pingpong, locals_for=(0,), device=DEV):
     ctx = binding.Odsgd(w, v, n_workers=wl.n_workers, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum,
                         wd=wl.wd, w_b=other if pingpong else None, w_delayed=None if pingpong else other,
                         local=local, tensor_offsets=wl.offsets,
-                        flags=binding.FLAG_DETERMINISTIC if det else 0)
+                        flags=binding.FLAG_DETERMINISTIC if det else binding.FLAG_ALLOW_FMA)
     return ctx, w, v, local
 
 

@@ -37,7 +37,7 @@ def _pair(wl, flags):
     return out
 
 
-@pytest.mark.parametrize("flags", [binding.FLAG_DETERMINISTIC, 0], ids=["deterministic", "default"])
+@pytest.mark.parametrize("flags", [0, binding.FLAG_ALLOW_FMA], ids=["default", "fma"])
 def test_static_table_call_matches_allocating_path_twice(cuda_device, flags):
     wl = W.workload("resnet56")  # 167 tensors in one launch
     (ref, v_ref, x_ref), (sta, v_sta, x_sta) = _pair(wl, flags)
