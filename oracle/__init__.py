@@ -48,6 +48,7 @@ def lib() -> ctypes.CDLL:
             "oracle_asgd_step": [f32p, sz, f32p, f32p, cf, cf, cf],
             "oracle_local_update_dc_c": [f32p, f32p, f32p, sz, f32p, cf, cf],
             "oracle_local_update_dc_a": [f32p, f32p, f32p, f32p, sz, f32p, cf, cf, cf, cf],
+            "oracle_local_update_momentum": [f32p, f32p, f32p, sz, f32p, cf, cf, cf],
             "oracle_global_update_mult": [pp32, ci, sz, f32p, f32p, f32p, cf, cf, cf,
                                           ctypes.POINTER(sz), sz, f32p, f32p],
             "oracle_dcasgd_step_c": [f32p, sz, f32p, f32p, cf, cf],
@@ -161,6 +162,19 @@ def local_update_dc_a(w_bak: np.ndarray, g: np.ndarray, x_prev: np.ndarray,
                                    _ptr(x_prev, ctypes.c_float),
                                    _ptr(mean_square, ctypes.c_float), n,
                                    _ptr(x, ctypes.c_float), local_lr, lam, m, eps)
+    return x
+
+
+def local_update_momentum(w_bak: np.ndarray, g: np.ndarray, u: np.ndarray, *, local_lr: float,
+                          momentum: float, wd: float, out: Optional[np.ndarray] = None) -> np.ndarray:
+    """Local SGD with momentum (Section 4.1's MNIST run); the velocity ``u`` is updated in place."""
+    n = _chk(w_bak, np.float32, "w_bak").shape[0]
+    _chk(g, np.float32, "g", n)
+    _chk(u, np.float32, "u", n)
+    x = np.empty(n, np.float32) if out is None else _chk(out, np.float32, "out", n)
+    lib().oracle_local_update_momentum(_ptr(w_bak, ctypes.c_float), _ptr(g, ctypes.c_float),
+                                       _ptr(u, ctypes.c_float), n, _ptr(x, ctypes.c_float),
+                                       local_lr, momentum, wd)
     return x
 
 

@@ -31,7 +31,8 @@
 //    compared to SSGD", i.e. the same rule as the global update.
 //  * ASGD step, Section 1 / 2.1: the server applies one worker's gradient as
 //    soon as it arrives (no sum, no 1/M).
-//  * DC-ASGD-c / DC-ASGD-a local updaters, Eq. 4, Eq. 5 and Eq. 6.
+//  * DC-ASGD-c / DC-ASGD-a local updaters, Eq. 4, Eq. 5 and Eq. 6; local SGD with momentum
+//    (Section 4.1's MNIST run); per-tensor multipliers; DC-ASGD at the server.
 //
 // Parity pins: every function here is pinned by tests/test_oracle_pins.py
 // (hand-worked dyadic example, closed forms on a diagonal quadratic, exact
@@ -153,6 +154,27 @@ int oracle_local_update_dc_a(const float* w_bak, const float* g, const float* x_
         const float d = g[i] + comp;
         const float step = local_lr * d;
         x[i] = w_bak[i] - step;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------- local SGD with momentum
+// Section 3.3 lets the local updater be any existing SGD-based algorithm, and the MNIST run
+// of Section 4.1 uses SGD with the same learning rate and momentum as the server.  That is
+// the server's own rule applied by worker m to its backup weights with its own gradient and
+// its own velocity u_m (one arena per worker):
+//   d = g + wd_l * w_bak;   u <- momentum_l * u - local_lr * d;   x = w_bak + u
+int oracle_local_update_momentum(const float* w_bak, const float* g, float* u, size_t n, float* x,
+                                 float local_lr, float momentum, float wd)
+{
+    for (size_t i = 0; i < n; ++i) {
+        const float decay = wd * w_bak[i];
+        const float d = g[i] + decay;
+        const float keep = momentum * u[i];
+        const float step = local_lr * d;
+        const float u_new = keep - step;
+        u[i] = u_new;
+        x[i] = w_bak[i] + u_new;
     }
     return 0;
 }

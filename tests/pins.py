@@ -48,6 +48,10 @@ class Impl:
         """returns (x, ms_new)"""
         raise NotImplementedError
 
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd) -> Tuple[np.ndarray, np.ndarray]:
+        """returns (x, u_new)"""
+        raise NotImplementedError
+
     def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult
                            ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
         """returns (w_new, v_new, w_prev)"""
@@ -468,6 +472,37 @@ def pin_multipliers(impl: Impl, seed: int = 66) -> None:
     np.testing.assert_array_equal(va[a:b], F32(mu) * v[a:b])
 
 
+# ----------------------------------------------------------------- local SGD with momentum
+
+def pin_local_momentum(impl: Impl, seed: int = 88) -> None:
+    """impl.local_update_momentum(w_bak, g, u, local_lr, momentum, wd) -> (x, u_new)"""
+    # the hand-worked server example, read as a local update: same rule, one gradient (gbar)
+    g = read_golden("worked_example_p8.txt")
+    gbar = a32((g["g0"] + g["g1"]) / 2)
+    x, u1 = impl.local_update_momentum(a32(g["w"]), gbar, a32(g["v"]), float(g["lr1"][0]),
+                                       float(g["momentum"][0]), float(g["wd"][0]))
+    assert np.array_equal(x, a32(g["w1"])) and np.array_equal(u1, a32(g["v1"]))
+    rng = np.random.default_rng(seed)
+    n = 400
+    w = a32(rng.normal(0, 1, n))
+    u = a32(rng.normal(0, 0.05, n))
+    gr = a32(rng.normal(0, 0.3, n))
+    # it IS the server's rule on one gradient: the ASGD step on (w_bak, u)
+    x, u1 = impl.local_update_momentum(w, gr, u.copy(), 0.07, 0.9, 2e-3)
+    wa, va = impl.asgd_step(gr, w.copy(), u.copy(), 0.07, 0.9, 2e-3)
+    assert_same_bits(x, wa, "local momentum rule vs the server rule on one gradient (weights)")
+    assert_same_bits(u1, va, "local momentum rule vs the server rule on one gradient (velocity)")
+    # no momentum, no decay: the plain compensation
+    x0, u0 = impl.local_update_momentum(w, gr, u.copy(), 0.07, 0.0, 0.0)
+    assert_same_bits(x0, impl.local_update(w, gr, 0.07), "momentum = wd = 0 reduces to x = w_bak - local_lr * g")
+    np.testing.assert_array_equal(u0, -(F32(0.07) * gr))
+    # the velocity carries over: two steps from u = 0 on a constant gradient move by (1 + (1 + mu)) * step
+    z = np.zeros(n, F32)
+    x1, ua = impl.local_update_momentum(w, gr, z, 0.5, 0.5, 0.0)
+    x2, ub = impl.local_update_momentum(x1, gr, ua, 0.5, 0.5, 0.0)
+    np.testing.assert_allclose(x2, w - 0.5 * gr * 2.5, rtol=0, atol=2e-6)
+
+
 # ----------------------------------------------------------------- DC-ASGD at the server
 
 def pin_dcasgd_server(impl: Impl, seed: int = 77) -> None:
@@ -517,4 +552,4 @@ CORE_PINS = (pin_worked_example, pin_rounding_order, pin_ssgd_quadratic_closed_f
              pin_odsgd_quadratic_matrix_form, pin_odsgd_special_cases, pin_invariants,
              pin_special_values, pin_exact_rational)
 DC_PINS = (pin_dc_worked_example, pin_dc_reductions)
-EXT_PINS = (pin_multipliers, pin_dcasgd_server)
+EXT_PINS = (pin_multipliers, pin_dcasgd_server, pin_local_momentum)

@@ -43,6 +43,11 @@ class OracleImpl(Impl):
         return x, ms
 
 
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd):
+        u = u.copy()
+        x = oracle.local_update_momentum(w_bak, g, u, local_lr=local_lr, momentum=momentum, wd=wd)
+        return x, u
+
     def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
         w, v = w.copy(), v.copy()
         wp = np.empty_like(w)
@@ -98,6 +103,10 @@ class NumpyImpl(Impl):
         lam_t = F32(lam) / np.sqrt(ms + F32(eps))
         return w_bak - F32(local_lr) * (g + (lam_t * (g * g)) * (w_bak - x_prev)), ms
 
+
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd):
+        x, un = self._server(g, w_bak, u, local_lr, momentum, wd)
+        return x, un
 
     def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
         gbar = self._sum(grads) * (F32(1.0) / F32(len(grads)))
@@ -383,6 +392,18 @@ class MultOnVelocityToo(NumpyImpl):
         return w + scale * vn, vn, wp
 
 
+class LocalMomentumFromNewVelocityOnly(NumpyImpl):
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd):
+        x, un = super().local_update_momentum(w_bak, g, u, local_lr, momentum, wd)
+        return w_bak - F32(local_lr) * g, un  # forgets the velocity in the weights
+
+
+class LocalMomentumDecayOnX(NumpyImpl):
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd):
+        x, un = super().local_update_momentum(w_bak, g, u, local_lr, momentum, 0.0)
+        return x - F32(local_lr) * F32(wd) * w_bak, un
+
+
 class DcasgdBackupNotRefreshed(NumpyImpl):
     def dcasgd_step_c(self, g, w, bak, lr, lam):
         return self.local_update_dc_c(w, g, bak, lr, lam), bak.copy()
@@ -399,7 +420,8 @@ class DcasgdRolesSwapped(NumpyImpl):
 
 
 @pytest.mark.parametrize("mutant", [MultSwapped, MultOffByOneTensor, MultOnVelocityToo, DcasgdBackupNotRefreshed,
-                                    DcasgdRolesSwapped], ids=lambda c: c.__name__)
+                                    DcasgdRolesSwapped, LocalMomentumFromNewVelocityOnly, LocalMomentumDecayOnX],
+                         ids=lambda c: c.__name__)
 def test_planted_ext_mistake_is_caught(mutant):
     assert _rejected_by(mutant(), pins.EXT_PINS), f"{mutant.__name__} slipped through"
 
