@@ -77,7 +77,7 @@ def parse_args():
     ap.add_argument("--block", type=int, default=0)
     ap.add_argument("--ctas-per-sm", type=int, default=0)
     ap.add_argument("--multipliers", action="store_true", help="per-tensor lr/wd multipliers (no decay off the weight tensors)")
-    ap.add_argument("--local-rule", choices=["sgd", "dc_c", "dc_a"], default="sgd")
+    ap.add_argument("--local-rule", choices=["sgd", "dc_c", "dc_a", "momentum"], default="sgd")
     ap.add_argument("--all-locals", action="store_true", help="update every worker's local weights in the fused pass")
     ap.add_argument("--sweep-workers", default="", help="comma list of worker counts (<= the workload's) to time as well")
     ap.add_argument("--graph", type=int, default=0,
@@ -222,10 +222,11 @@ def run_cuda(args):
     stream = torch.cuda.current_stream()
     extra_streams = 0  # arenas touched per local update beyond the plain rule's single store
     if args.local_rule != "sgd":
-        rule = binding.LOCAL_DC_C if args.local_rule == "dc_c" else binding.LOCAL_DC_A
-        ms = [torch.zeros_like(w_a) for _ in range(n_locals)] + [None] * (M - n_locals) if rule == binding.LOCAL_DC_A else None
-        ctx.set_local_rule(rule, 0.04, 0.95, 1e-7, ms)
-        extra_streams = n_locals * (1 if rule == binding.LOCAL_DC_C else 3)  # x_prev read (+ mean square read, write)
+        rule = {"dc_c": binding.LOCAL_DC_C, "dc_a": binding.LOCAL_DC_A, "momentum": binding.LOCAL_MOMENTUM}[args.local_rule]
+        ms = [torch.zeros_like(w_a) for _ in range(n_locals)] + [None] * (M - n_locals) if rule != binding.LOCAL_DC_C else None
+        ctx.set_local_rule(rule, 0.04 if rule != binding.LOCAL_MOMENTUM else wl.wd, 0.95, 1e-7, ms)
+        # arenas touched per local update beyond the store of x: x_prev read (Eq. 4, 5), state read + write
+        extra_streams = n_locals * {binding.LOCAL_DC_C: 1, binding.LOCAL_DC_A: 3, binding.LOCAL_MOMENTUM: 2}[rule]
     if args.multipliers:
         ctx.set_tensor_multipliers(None, [1.0 if t.kind == "weight" else 0.0 for t in wl.tensors])
 

@@ -78,6 +78,7 @@ extern "C" {
 #define ODSGD_LOCAL_SGD 0  /* x = w_bak - local_lr * g */
 #define ODSGD_LOCAL_DC_C 1 /* Eq. 4 */
 #define ODSGD_LOCAL_DC_A 2 /* Eq. 5 with the running mean square of Eq. 6 */
+#define ODSGD_LOCAL_MOMENTUM 3 /* the server's own rule run by the worker: SGD with momentum (and decay) */
 
 typedef struct odsgd_ctx odsgd_ctx;
 
@@ -210,7 +211,13 @@ int odsgd_set_wd(odsgd_ctx* ctx, float wd);
  * n_workers device pointers (n_params floats each, caller-owned and caller-initialised,
  * normally zeros; entries may be NULL for workers that are never updated locally, and the
  * whole table may be NULL when the rule is only used by odsgd_dcasgd_step); pass NULL for
- * the other rules.  A local update of a worker without its arena fails with ERR_STATE.  In both delay-compensated rules the vector the
+ * the other rules.  A local update of a worker without its arena fails with ERR_STATE.
+ * ODSGD_LOCAL_MOMENTUM (Section 4.1's MNIST run: local SGD with the server's learning rate and
+ * momentum) applies the global update's rule to the worker's backup weights, its own gradient
+ * and its own velocity:  d = g + lambda * w_bak;  u <- m * u - local_lr * d;  x = w_bak + u,
+ * with `m` the local momentum, `lambda` the local weight decay, `eps` unused, and
+ * `mean_square` holding the per-worker velocity arenas u (same rules as above, zero-filled
+ * for a fresh run).  In both delay-compensated rules the vector the
  * gradient was computed on (the paper's w_t) is the worker's previous local weights,
  * i.e. the content of local[worker] before the call, which is then overwritten.
  */

@@ -21,7 +21,7 @@ MAX_WORKERS = 64
 FLAG_DETERMINISTIC = 0x1
 FLAG_ALLOW_UNALIGNED = 0x2
 FLAG_ALLOW_FMA = 0x4
-LOCAL_SGD, LOCAL_DC_C, LOCAL_DC_A = 0, 1, 2
+LOCAL_SGD, LOCAL_DC_C, LOCAL_DC_A, LOCAL_MOMENTUM = 0, 1, 2, 3
 
 OK, ERR_ARG, ERR_ALIGN, ERR_OVERLAP, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 

@@ -194,6 +194,7 @@ int launch_server_r(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
     switch (c->local_rule) {
         case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, st);
         case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, st);
+        case ODSGD_LOCAL_MOMENTUM: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_MOMENTUM>(c, a, st);
         default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, st);
     }
 }
@@ -236,6 +237,7 @@ int launch_local_r(odsgd_ctx* c, const LocalArgs& a, bool server, cudaStream_t s
     switch (c->local_rule) {
         case ODSGD_LOCAL_SGD: return launch_local_t<DET, NL, ODSGD_LOCAL_SGD, false>(c, a, st);
         case ODSGD_LOCAL_DC_C: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_C, false>(c, a, st);
+        case ODSGD_LOCAL_MOMENTUM: return launch_local_t<DET, NL, ODSGD_LOCAL_MOMENTUM, false>(c, a, st);
         default: return launch_local_t<DET, NL, ODSGD_LOCAL_DC_A, false>(c, a, st);
     }
 }
@@ -305,7 +307,7 @@ int check_grads(odsgd_ctx* c, const float* const* grads, std::vector<Named>* ptr
 // Local mode and outputs for a fused call; fills a.x / a.ms / a.local_worker.
 int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mode, std::vector<Named>* ptrs) {
     if (worker_id >= c->n_workers || worker_id < -1) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
-    const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
+    const bool need_ms = needs_state(c->local_rule);
     if (worker_id >= 0) {
         if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
         if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for that worker");
@@ -523,8 +525,8 @@ int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     if (!c->grads_bound) return fail(c, ODSGD_ERR_STATE, "no gradients bound: call odsgd_global_update first");
     if (!c->delayed) return fail(c, ODSGD_ERR_STATE, "this context keeps no backup weights (in-place layout without w_delayed)");
     if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
-    const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
-    if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for that worker");
+    const bool need_ms = needs_state(c->local_rule);
+    if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no state arena (mean square / velocity) for that worker");
     LocalArgs a;
     a.w_bak = c->delayed;
     a.g = c->bound[worker_id];
@@ -642,9 +644,9 @@ int odsgd_set_wd(odsgd_ctx* ctx, float wd) {
 int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float eps, float* const* mean_square) {
     if (!ctx) return ODSGD_ERR_ARG;
     odsgd_ctx* c = ctx;
-    if (rule != ODSGD_LOCAL_SGD && rule != ODSGD_LOCAL_DC_C && rule != ODSGD_LOCAL_DC_A)
+    if (rule != ODSGD_LOCAL_SGD && rule != ODSGD_LOCAL_DC_C && rule != ODSGD_LOCAL_DC_A && rule != ODSGD_LOCAL_MOMENTUM)
         return fail(c, ODSGD_ERR_ARG, "unknown local rule");
-    if (rule == ODSGD_LOCAL_DC_A && mean_square) {
+    if (needs_state(rule) && mean_square) {
         odsgd_ctx probe = *c;
         for (int w = 0; w < c->n_workers; ++w) probe.mean_square[w] = mean_square[w];
         const std::vector<Named> st = state_buffers(&probe);

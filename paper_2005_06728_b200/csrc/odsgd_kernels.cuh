@@ -245,11 +245,23 @@ __device__ __forceinline__ void server_rule(float gbar, float w, float v, float 
 
 // Local updater on one element (Section 3.3).  x_prev / ms are only touched by
 // the delay-compensated rules.
+// Which extra arenas a local rule touches: the worker's previous local weights (Eq. 4, Eq. 5)
+// and a per-worker state arena (Eq. 6's mean square, or the velocity of local momentum SGD).
+__host__ __device__ constexpr bool needs_prev(int rule) { return rule == ODSGD_LOCAL_DC_C || rule == ODSGD_LOCAL_DC_A; }
+__host__ __device__ constexpr bool needs_state(int rule) { return rule == ODSGD_LOCAL_DC_A || rule == ODSGD_LOCAL_MOMENTUM; }
+
 template <bool DET, int RULE>
 __device__ __forceinline__ float local_rule(float w_bak, float g, float x_prev, float& ms, const LocalParams& p) {
     using O = Op<DET>;
     if (RULE == ODSGD_LOCAL_SGD) {
         return O::sub(w_bak, O::mul(p.local_lr, g));
+    }
+    if (RULE == ODSGD_LOCAL_MOMENTUM) {
+        // the server's rule run by the worker: state = velocity, m = local momentum, lambda = local decay
+        float x, u;
+        server_rule<DET>(g, w_bak, ms, p.local_lr, p.m, p.lambda, x, u);
+        ms = u;
+        return x;
     }
     const float gg = O::mul(g, g);
     float lam = p.lambda;
@@ -323,8 +335,8 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
                             if (ok[u]) {
-                                xv[j][u] = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
-                                if (RULE == ODSGD_LOCAL_DC_A) msv[j][u] = load_stream<NL>(a.ms[m0 + j] + off[u]);
+                                if (needs_prev(RULE)) xv[j][u] = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+                                if (needs_state(RULE)) msv[j][u] = load_stream<NL>(a.ms[m0 + j] + off[u]);
                             }
                         }
                     }
@@ -358,7 +370,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                                                                     msv[j][u].e[l], a.lp);
                                 }
                                 store_stream<NL>(xp + off[u], xo);
-                                if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[m] + off[u], msv[j][u]);
+                                if (needs_state(RULE)) store_stream<NL>(a.ms[m] + off[u], msv[j][u]);
                             }
                         }
                     }
@@ -384,14 +396,14 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
         if (LOCAL == kLocalOne) {
             float* xp = a.x[0];
             Vec<NL> xo, xv, msv;
-            if (RULE != ODSGD_LOCAL_SGD) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
-            if (RULE == ODSGD_LOCAL_DC_A) msv = load_stream<NL>(a.ms[0] + off[u]);
+            if (needs_prev(RULE)) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+            if (needs_state(RULE)) msv = load_stream<NL>(a.ms[0] + off[u]);
 #pragma unroll
             for (int l = 0; l < NL; ++l) {
                 xo.e[l] = local_rule<DET, RULE>(w[u].e[l], gl[u].e[l], xv.e[l], msv.e[l], a.lp);
             }
             store_stream<NL>(xp + off[u], xo);
-            if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms[0] + off[u], msv);
+            if (needs_state(RULE)) store_stream<NL>(a.ms[0] + off[u], msv);
         }
         if (a.w_prev != nullptr) store_stream<NL>(a.w_prev + off[u], w[u]);
         store_stream<NL>(a.v + off[u], vn);
@@ -449,8 +461,8 @@ __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned
         if (ok[u]) {
             w[u] = SERVER ? load_stream<NL>(a.w_bak + off[u]) : load_grad<NL>(a.w_bak + off[u]);
             g[u] = load_grad<NL>(a.g + off[u]);
-            if (RULE != ODSGD_LOCAL_SGD) xv[u] = a.lp.first ? w[u] : load_stream<NL>(a.x + off[u]);
-            if (RULE == ODSGD_LOCAL_DC_A) msv[u] = load_stream<NL>(a.ms + off[u]);
+            if (needs_prev(RULE)) xv[u] = a.lp.first ? w[u] : load_stream<NL>(a.x + off[u]);
+            if (needs_state(RULE)) msv[u] = load_stream<NL>(a.ms + off[u]);
         }
     }
 #pragma unroll
@@ -461,7 +473,7 @@ __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned
         for (int l = 0; l < NL; ++l) xo.e[l] = local_rule<DET, RULE>(w[u].e[l], g[u].e[l], xv[u].e[l], msv[u].e[l], a.lp);
         store_stream<NL>(a.x + off[u], xo);
         if (SERVER) store_stream<NL>(a.w_out + off[u], xo);
-        if (RULE == ODSGD_LOCAL_DC_A) store_stream<NL>(a.ms + off[u], msv[u]);
+        if (needs_state(RULE)) store_stream<NL>(a.ms + off[u], msv[u]);
     }
 }
 

@@ -151,6 +151,9 @@ class GpuImpl(Impl):
         return self._local(w_bak, g, local_lr, binding.LOCAL_DC_A, x_prev=x_prev, ms=ms, lam=lam, m=m, eps=eps)
 
 
+    def local_update_momentum(self, w_bak, g, u, local_lr, momentum, wd):
+        return self._local(w_bak, g, local_lr, binding.LOCAL_MOMENTUM, ms=u, lam=wd, m=momentum)
+
     def global_update_mult(self, grads, w, v, lr, momentum, wd, offsets, lr_mult, wd_mult):
         self.bufs = []
         wa, b0 = dev_arena(w)

@@ -117,11 +117,13 @@ def _dc_oracle_local(rule, wp, g, x_prev, ms, llr, lam, m, eps):
         return oracle.local_update(wp, g, local_lr=llr)
     if rule == binding.LOCAL_DC_C:
         return oracle.local_update_dc_c(wp, g, x_prev, local_lr=llr, lam=lam)
+    if rule == binding.LOCAL_MOMENTUM:
+        return oracle.local_update_momentum(wp, g, ms, local_lr=llr, momentum=m, wd=lam)
     return oracle.local_update_dc_a(wp, g, x_prev, ms, local_lr=llr, lam=lam, m=m, eps=eps)
 
 
-@pytest.mark.parametrize("rule", [binding.LOCAL_SGD, binding.LOCAL_DC_C, binding.LOCAL_DC_A],
-                         ids=["sgd", "dc_c", "dc_a"])
+@pytest.mark.parametrize("rule", [binding.LOCAL_SGD, binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
+                         ids=["sgd", "dc_c", "dc_a", "momentum"])
 @pytest.mark.parametrize("wp", [0, 1, 3])
 def test_algorithm2_state_machine(cuda_device, rule, wp):
     """odsgd_step: wp SSGD iterations, then fused global + local updates; the first local
@@ -136,7 +138,8 @@ def test_algorithm2_state_machine(cuda_device, rule, wp):
     msq = [torch.zeros_like(w) for _ in range(M)]
     ctx = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
                         w_b=w_b, local=local, tensor_offsets=wl.offsets, flags=binding.FLAG_DETERMINISTIC)
-    ctx.set_local_rule(rule, lam, m_, eps, msq if rule == binding.LOCAL_DC_A else None)
+    has_state = rule in (binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM)
+    ctx.set_local_rule(rule, lam, m_, eps, msq if has_state else None)
     ctx.set_warmup(wp)
     w_ref, v_ref = w.cpu().numpy().copy(), v.cpu().numpy().copy()
     x_ref = [None] * M
@@ -166,14 +169,15 @@ def test_algorithm2_state_machine(cuda_device, rule, wp):
         if k >= wp:
             for mm in range(M):
                 assert_bits(local[mm].cpu().numpy(), x_ref[mm], f"x[{mm}] at iteration {k}")
-                if rule == binding.LOCAL_DC_A:
-                    assert_bits(msq[mm].cpu().numpy(), ms_ref[mm], f"mean square [{mm}] at iteration {k}")
+                if has_state:
+                    assert_bits(msq[mm].cpu().numpy(), ms_ref[mm], f"state arena [{mm}] at iteration {k}")
     with pytest.raises(binding.OdsgdError) as e:
         ctx.set_warmup(5)
     assert e.value.code == binding.ERR_STATE
 
 
-@pytest.mark.parametrize("rule", [binding.LOCAL_DC_C, binding.LOCAL_DC_A], ids=["dc_c", "dc_a"])
+@pytest.mark.parametrize("rule", [binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
+                         ids=["dc_c", "dc_a", "momentum"])
 def test_separate_dc_local_update_equals_fused(cuda_device, rule):
     wl = W.ragged_workload([10_000, 33], n_workers=2)
     ctxs = []
@@ -184,7 +188,7 @@ def test_separate_dc_local_update_equals_fused(cuda_device, rule):
         ms = [torch.zeros_like(w), torch.zeros_like(w)]
         c = binding.Odsgd(w, v, n_workers=2, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
                           w_b=torch.zeros_like(w), local=local, flags=binding.FLAG_DETERMINISTIC)
-        c.set_local_rule(rule, 0.3, 0.9, 1e-6, ms if rule == binding.LOCAL_DC_A else None)
+        c.set_local_rule(rule, 0.3, 0.9, 1e-6, ms if rule != binding.LOCAL_DC_C else None)
         ctxs.append((c, v, local, ms))
     for it in range(3):
         grads = W.make_grads(wl, it, DEV)
@@ -197,7 +201,7 @@ def test_separate_dc_local_update_equals_fused(cuda_device, rule):
             assert torch.equal(ctxs[0][2][m], ctxs[1][2][m]) and torch.equal(ctxs[0][3][m], ctxs[1][3][m])
         assert torch.equal(ctxs[0][0].weights(), ctxs[1][0].weights())
     # a worker without its mean-square arena cannot be updated under DC_A
-    if rule == binding.LOCAL_DC_A:
+    if rule != binding.LOCAL_DC_C:
         c = ctxs[0][0]
         c.set_local_rule(rule, 0.3, 0.9, 1e-6, [ctxs[0][3][0], None])
         with pytest.raises(binding.OdsgdError) as e:
