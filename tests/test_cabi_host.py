@@ -172,3 +172,32 @@ def test_lr_schedules_match_their_closed_forms(lib):
     assert all(a <= b for a, b in zip(ramp, ramp[1:])) and ramp[0] == f32(0.1) and ramp[-1] == f32(0.8)
     poly = [binding.odsgd_lr_poly_decay(0.4, 0.0, 2.0, 100, k) for k in range(0, 120)]
     assert all(a >= b for a, b in zip(poly, poly[1:])) and poly[-1] == 0.0
+
+
+def test_header_is_plain_c_and_links_from_a_c_program(lib, tmp_path):
+    """include/odsgd.h compiles as C99 with all warnings on, and a C program linked against
+    libodsgd.so can call into it (no C++ or torch types at the boundary)."""
+    import shutil
+    import subprocess
+
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not available")
+    src = tmp_path / "use_odsgd.c"
+    src.write_text(
+        '#include <stdio.h>\n#include "odsgd.h"\n'
+        "int main(void) {\n"
+        "    odsgd_ctx* ctx = (odsgd_ctx*)1;\n"
+        "    odsgd_desc d = {0};\n"
+        "    int rc = odsgd_create(&ctx, &d);\n"
+        '    printf("%d %d %d %s\\n", odsgd_version(), rc, ctx == NULL, odsgd_strerror(rc));\n'
+        "    return (rc == ODSGD_ERR_ARG && ctx == NULL) ? 0 : 1;\n"
+        "}\n")
+    exe = tmp_path / "use_odsgd"
+    pkg = os.path.join(ROOT, "paper_2005_06728_b200")
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", f"-I{os.path.join(ROOT, 'include')}",
+           str(src), "-o", str(exe), f"-L{pkg}", "-lodsgd", f"-Wl,-rpath,{pkg}"]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    assert res.returncode == 0, res.stderr
+    run = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert run.returncode == 0, run.stdout + run.stderr
+    assert run.stdout.split()[:3] == ["1", str(binding.ERR_ARG), "1"]
