@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <new>
 #include <string>
 #include <vector>
@@ -50,6 +51,8 @@ struct odsgd_ctx {
     cudaEvent_t ev_kernel_done = nullptr;  // recorded on the compute stream after the update kernel
     cudaEvent_t ev_copy_done = nullptr;    // recorded on the copy stream after the device-to-host copy
     bool copy_pending = false;
+    // resident CTAs per SM by (kernel, block size); 0 = that block size cannot be launched
+    std::map<std::pair<const void*, int>, int> occupancy;
     std::string err;
 };
 
@@ -153,6 +156,28 @@ int resident_ctas(K kernel, int block) {
     return n;
 }
 
+// Cached per context (a context belongs to one device and is used from one thread at a time).
+template <typename K>
+int resident_cached(odsgd_ctx* c, K kernel, int block) {
+    const std::pair<const void*, int> key(reinterpret_cast<const void*>(kernel), block);
+    auto it = c->occupancy.find(key);
+    if (it != c->occupancy.end()) return it->second;
+    const int n = resident_ctas(kernel, block);
+    c->occupancy[key] = n;
+    return n;
+}
+
+// Every launching call runs on the device the context was created on.
+int on_own_device(odsgd_ctx* c) {
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("cudaGetDevice: ") + cudaGetErrorString(e));
+    if (dev != c->device)
+        return fail(c, ODSGD_ERR_STATE, "the current CUDA device (" + std::to_string(dev) + ") is not the one the context was created on (" +
+                                            std::to_string(c->device) + ")");
+    return ODSGD_OK;
+}
+
 int too_wide(odsgd_ctx* c, int block) {
     return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
 }
@@ -161,12 +186,7 @@ template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
     auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT, BB, UB>;
-    static int cached_block = 0, cached_res = 0;
-    if (cached_block != block) {
-        cached_res = resident_ctas(kernel, block);
-        cached_block = block;
-    }
-    if (cached_res == 0) return too_wide(c, block);
+    if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     const int grid = grid_for(c, a.n, NL, block, UB, kServerCtasPerSm);
     kernel<<<grid, block, 0, st>>>(a);
     return after_launch(c, "server kernel launch");
@@ -218,12 +238,7 @@ template <bool DET, int NL, int RULE, bool SERVER>
 int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = local_kernel<DET, NL, RULE, SERVER>;
-    static int cached_block = 0, cached_res = 0;
-    if (cached_block != block) {
-        cached_res = resident_ctas(kernel, block);
-        cached_block = block;
-    }
-    if (cached_res == 0) return too_wide(c, block);
+    if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
     return after_launch(c, "local kernel launch");
 }
@@ -252,12 +267,7 @@ template <bool DET, int NL>
 int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = asgd_kernel<DET, NL>;
-    static int cached_block = 0, cached_res = 0;
-    if (cached_block != block) {
-        cached_res = resident_ctas(kernel, block);
-        cached_block = block;
-    }
-    if (cached_res == 0) return too_wide(c, block);
+    if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
     return after_launch(c, "asgd kernel launch");
 }
@@ -279,9 +289,12 @@ LocalParams local_params(const odsgd_ctx* c) {
     return p;
 }
 
-// A copy-back of local weights that odsgd_fused_update_host put on a separate copy stream
-// must be out before any later kernel overwrites a local arena: make `st` wait for it.
-int settle_copy(odsgd_ctx* c, cudaStream_t st) {
+// Run before every kernel launch: the context's device must be current, and a copy-back of
+// local weights that odsgd_fused_update_host put on a separate copy stream must be out before
+// a later kernel overwrites a local arena (`st` is made to wait for it).
+int before_launch(odsgd_ctx* c, cudaStream_t st) {
+    const int rc_dev = on_own_device(c);
+    if (rc_dev != ODSGD_OK) return rc_dev;
     if (!c->copy_pending) return ODSGD_OK;
     const cudaError_t e = cudaStreamWaitEvent(st, c->ev_copy_done, 0);
     if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("stream wait: ") + cudaGetErrorString(e));
@@ -398,7 +411,7 @@ int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
             if (o % 4 != 0) { lanes = 1; break; }
     }
 
-    rc = settle_copy(c, static_cast<cudaStream_t>(stream));
+    rc = before_launch(c, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
     rc = launch_server(c, a, lanes, local_mode, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
@@ -539,7 +552,7 @@ int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     if (need_ms) ptrs.push_back({a.ms, "mean_square", worker_id});
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
-    const int rc_copy = settle_copy(c, static_cast<cudaStream_t>(stream));
+    const int rc_copy = before_launch(c, static_cast<cudaStream_t>(stream));
     if (rc_copy != ODSGD_OK) return rc_copy;
     return launch_local(c, a, lanes, false, static_cast<cudaStream_t>(stream));
 }
@@ -609,6 +622,8 @@ int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stre
     a.wd = c->wd;
     const int lanes = lanes_for(c, {g, {a.w, "w", -1}, {a.v, "v", -1}});
     if (lanes == 0) return ODSGD_ERR_ALIGN;
+    const int rc_dev = on_own_device(c);
+    if (rc_dev != ODSGD_OK) return rc_dev;
     const int rc = launch_asgd(c, a, lanes, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
     c->step += 1;
@@ -750,7 +765,7 @@ int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* st
     if (need_ms) ptrs.push_back({a.ms, "server_mean_square", -1});
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
-    const int rc_copy = settle_copy(c, static_cast<cudaStream_t>(stream));
+    const int rc_copy = before_launch(c, static_cast<cudaStream_t>(stream));
     if (rc_copy != ODSGD_OK) return rc_copy;
     const int rc = launch_local(c, a, lanes, true, static_cast<cudaStream_t>(stream));
     if (rc != ODSGD_OK) return rc;
@@ -986,7 +1001,7 @@ int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_gr
     a.t_wd_mult = a.t_lr_mult + nt;
     a.n_tensors = (unsigned int)nt;
 
-    rc = settle_copy(c, st);
+    rc = before_launch(c, st);
     if (rc != ODSGD_OK) return rc;
     const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
     if (det)
