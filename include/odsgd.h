@@ -73,6 +73,10 @@ extern "C" {
 #define ODSGD_FLAG_DETERMINISTIC 0x1u   /* one rounding per operator; this is the default, the bit only states it */
 #define ODSGD_FLAG_ALLOW_UNALIGNED 0x2u /* accept 4-byte aligned pointers (slower scalar kernel) */
 #define ODSGD_FLAG_ALLOW_FMA 0x4u       /* let multiply-add pairs fuse (excludes ODSGD_FLAG_DETERMINISTIC) */
+#define ODSGD_FLAG_WORKER_ONLY 0x8u     /* worker-role context: v may be NULL; only odsgd_worker_local_update runs */
+
+/* Gradient tables one context can keep bound at a time (odsgd_bind_grads). */
+#define ODSGD_MAX_BINDINGS 16
 
 /* Local update rules (Section 3.3, "Local Updater"). */
 #define ODSGD_LOCAL_SGD 0  /* x = w_bak - local_lr * g */
@@ -101,7 +105,8 @@ typedef struct odsgd_desc {
     float* w_a;                   /* device, n_params floats: global weights w_0 at create time */
     float* w_b;                   /* device, n_params floats, or NULL */
     float* w_delayed;             /* device, n_params floats, or NULL (in-place layout only) */
-    float* v;                     /* device, n_params floats: momentum state (caller zero-fills for a fresh run) */
+    float* v;                     /* device, n_params floats: momentum state (caller zero-fills for a fresh run);
+                                     may be NULL only with ODSGD_FLAG_WORKER_ONLY */
     float* const* local;          /* host array of n_workers device pointers (entries may be NULL), or NULL */
     size_t n_params;              /* elements in each arena, > 0 */
     const size_t* tensor_offsets; /* host, n_tensors + 1 ascending offsets, [0] = 0, [n_tensors] = n_params */
@@ -177,7 +182,10 @@ int odsgd_fused_update(odsgd_ctx* ctx, const float* const* worker_grads, int wor
  * overlaps the NEXT call's uploads (the bus is full duplex); the next call's kernel waits for
  * that copy before it overwrites local[worker_id].  The caller synchronises `copy_stream`
  * before reading `host_local_out`.  (The context creates two CUDA events on first use of a
- * separate copy stream.)
+ * separate copy stream.)  Every check that can refuse the call runs before the first copy is
+ * enqueued, so a failed call leaves `dev_staging` untouched; and every later kernel this
+ * context launches that may write a local arena, on whatever stream, first waits for a
+ * copy-back that is still pending.
  */
 int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, float* const* dev_staging,
                             int worker_id, float* host_local_out, void* stream, void* copy_stream);
@@ -197,7 +205,73 @@ int odsgd_ssgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stre
  */
 int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream);
 
-/* Hyper-parameters are kernel arguments, so schedules may change them before any call. */
+/*
+ * The same three server calls on a gradient table that was checked once.  A training loop
+ * hands the library the same M gradient buffers every iteration; odsgd_bind_grads() validates
+ * such a table (NULL entries, overlap with every state buffer, alignment) and keeps a copy of
+ * its pointers in one of ODSGD_MAX_BINDINGS slots of the context, and the *_bound calls then
+ * skip that validation: their per-call host work is filling the kernel's argument block and the
+ * launch.  (Algorithm 1 and Algorithm 2 run once per iteration on the same buffers; on small
+ * parameter sets the host side of a call, not the kernel, is what bounds the iteration rate.)
+ * Results are bit-identical to the unbound calls.
+ *   odsgd_bind_grads    worker_grads as in odsgd_global_update; *slot receives the slot index.
+ *                       Errors: ERR_ARG, ERR_OVERLAP, ERR_ALIGN as that call would report them,
+ *                       ERR_UNSUPPORTED when all slots are taken; *slot is then -1.
+ *   odsgd_unbind_grads  frees a slot.
+ *   *_bound             ERR_ARG for a slot that holds no table; ERR_STATE when the context's set
+ *                       of state buffers changed after the bind (odsgd_set_local_rule,
+ *                       odsgd_set_server_mean_square): the table must be bound again, which
+ *                       repeats the overlap check against the new buffers.  Otherwise the errors
+ *                       of the unbound call.
+ * The bound buffers must stay valid, and must keep not overlapping the state, for as long as the
+ * slot is used; the library cannot see a buffer being freed and reallocated elsewhere.
+ */
+int odsgd_bind_grads(odsgd_ctx* ctx, const float* const* worker_grads, int* slot);
+int odsgd_unbind_grads(odsgd_ctx* ctx, int slot);
+int odsgd_global_update_bound(odsgd_ctx* ctx, int slot, void* stream);
+int odsgd_fused_update_bound(odsgd_ctx* ctx, int slot, int worker_id, void* stream);
+int odsgd_ssgd_step_bound(odsgd_ctx* ctx, int slot, void* stream);
+
+/*
+ * The worker's half of an iteration when the server's half runs elsewhere (Algorithm 2,
+ * repeat-loop: "w_bak = w_t", then "Update w_bak with g_m", while the gradient is on its way to
+ * the server; Section 3.1: push and local update overlap because both only read the gradient).
+ * Applies the context's local rule to explicit inputs:
+ *     local[worker_id] = LocalRule(w_bak, grad)        (x = w_bak - local_lr * grad by default)
+ * `w_bak`: device, n_params floats, the global weights this worker pulled last; it may be one of
+ * the context's own weight arenas (w_a / w_b), but not an arena the call writes.  `grad`: device,
+ * n_params floats, this worker's gradient, outside every state buffer.  `no_delay` != 0 says
+ * that `grad` was computed on `w_bak` itself (the last warm-up iteration of Algorithm 2), so the
+ * delay-compensated rules of Eq. 4 / Eq. 5 see a zero delay; it is ignored by the other rules.
+ * Works in any context; a context created with ODSGD_FLAG_WORKER_ONLY (no momentum arena) can
+ * run nothing else: its server calls fail with ERR_STATE.  Does not touch the step counter or
+ * the weights.
+ * Errors: ERR_ARG, ERR_OVERLAP, ERR_ALIGN, ERR_STATE (rule needs a state arena the worker lacks).
+ */
+int odsgd_worker_local_update(odsgd_ctx* ctx, int worker_id, const float* w_bak, const float* grad,
+                              int no_delay, void* stream);
+
+/*
+ * Which slice of the arena rank `rank` of `n_ranks` owns when the server role is spread over
+ * several GPUs (Section 2.2: gradients are reduced, pushed to the server and the new weights
+ * pulled back; every element is updated independently, so the server's work shards by index).
+ * All slices have the same nominal length, ceil(n_params / n_ranks) rounded up to 4 elements
+ * (16 bytes, so every slice start keeps the arena's alignment); slice r is
+ * [r * len, min((r + 1) * len, n_params)).  The slices are disjoint, ascending and cover
+ * [0, n_params) exactly; the last non-empty one may be short, and with more ranks than
+ * 4-element groups the trailing ranks get empty slices (begin == end == n_params).
+ * Host arithmetic only.  Errors: ERR_ARG (NULL output, n_ranks < 1, rank out of range).
+ */
+int odsgd_shard_range(size_t n_params, int n_ranks, int rank, size_t* begin, size_t* end);
+
+/*
+ * Hyper-parameters are kernel arguments, never compiled in: the paper's runs change the
+ * learning rates during training (Section 4: division by 10 at fixed epochs, the linear ramp
+ * from 0.1 to 0.8 over the first epochs, polynomial decay; global and local rates are chosen
+ * separately, Section 4.2), so a setter may be called before any update call and takes effect
+ * from the next launch on.  Momentum and weight decay are the server rule's (Section 4.1:
+ * momentum 0.9 for SSGD and OD-SGD, 0 for ASGD).
+ */
 int odsgd_set_lr(odsgd_ctx* ctx, float lr);
 int odsgd_set_local_lr(odsgd_ctx* ctx, float local_lr);
 int odsgd_set_momentum(odsgd_ctx* ctx, float momentum);
@@ -261,12 +335,18 @@ int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const flo
  * launched); local rule ODSGD_LOCAL_SGD only (else ERR_UNSUPPORTED); tensor offsets must be
  * multiples of 4 elements unless ODSGD_FLAG_ALLOW_UNALIGNED is set (ERR_ALIGN).
  * Set-up: the first call on each device looks up the array's device address
- * (cudaGetSymbolAddress) with that device current; make that first call outside any stream
- * capture.  Sharing: every call on a device, from every context, writes the same array, and
+ * (cudaGetSymbolAddress) with that device current.  The call cannot be recorded into a stream
+ * capture: while `stream` is capturing it fails with ERR_STATE and enqueues nothing (a captured
+ * upload would re-read, at every replay, whatever table the last eager call left behind).
+ * Sharing: every call on a device, from every context, writes the same array, and
  * the array keeps the last call's table.  Each call rewrites all entries it uses before its
  * kernel reads them, in stream order, so calls on ONE stream are safe back to back; calls
  * whose work overlaps on the GPU (different streams, different threads) race on the array
- * and must be serialised by the caller.
+ * and must be serialised by the caller.  On the host the table is staged in one pageable array
+ * shared by the whole process; the call holds a process-wide lock while it fills and uploads
+ * it, so host threads may call concurrently (also for different devices), at the price of
+ * running one at a time.  The upload is an ordinary copy from pageable memory: for a large
+ * table it may make the call wait for work enqueued earlier on `stream`.
  */
 #define ODSGD_STATIC_MAX_TENSORS 4096
 #define ODSGD_STATIC_TABLE_BYTES (16 * ODSGD_STATIC_MAX_TENSORS + 8)
@@ -307,6 +387,7 @@ int odsgd_set_server_mean_square(odsgd_ctx* ctx, float* mean_square);
  */
 int odsgd_set_warmup(odsgd_ctx* ctx, uint64_t wp);
 int odsgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream);
+int odsgd_step_bound(odsgd_ctx* ctx, int slot, void* stream); /* the same on a table bound by odsgd_bind_grads */
 int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights);
 
 /*
@@ -336,7 +417,9 @@ float odsgd_lr_poly_decay(float base_lr, float end_lr, float power, uint64_t tot
  * *delayed is NULL when the context keeps no backup or none is valid yet. */
 int odsgd_get_weights(odsgd_ctx* ctx, float** current, float** delayed);
 
-/* Number of global updates (OD-SGD or SSGD) plus ASGD steps applied so far. */
+/* Number of global updates (OD-SGD or SSGD) plus ASGD / DC-ASGD steps applied so far: the
+ * server's counter t of Algorithm 1 ("t <- t + 1" after each update of w_t).  The setter is for
+ * resuming from a checkpoint. */
 int odsgd_get_step(odsgd_ctx* ctx, uint64_t* step);
 int odsgd_set_step(odsgd_ctx* ctx, uint64_t step);
 

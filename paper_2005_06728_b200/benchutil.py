@@ -8,7 +8,6 @@ import os
 import statistics
 import subprocess
 import threading
-import time
 from typing import Dict, List, Optional
 
 BAD_REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
@@ -218,7 +217,3 @@ def host_info() -> Dict:
     except OSError:
         pass
     return {"nproc": os.cpu_count(), "cpu": model}
-
-
-def now() -> float:
-    return time.perf_counter()

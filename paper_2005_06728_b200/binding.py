@@ -21,6 +21,8 @@ MAX_WORKERS = 64
 FLAG_DETERMINISTIC = 0x1
 FLAG_ALLOW_UNALIGNED = 0x2
 FLAG_ALLOW_FMA = 0x4
+FLAG_WORKER_ONLY = 0x8
+MAX_BINDINGS = 16
 LOCAL_SGD, LOCAL_DC_C, LOCAL_DC_A, LOCAL_MOMENTUM = 0, 1, 2, 3
 
 OK, ERR_ARG, ERR_ALIGN, ERR_OVERLAP, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
@@ -35,6 +37,8 @@ EXPORTS = (
     "odsgd_set_tensor_multipliers", "odsgd_dcasgd_step", "odsgd_set_server_mean_square", "odsgd_set_warmup",
     "odsgd_step", "odsgd_get_train_weights", "odsgd_lr_step_decay", "odsgd_lr_linear_ramp",
     "odsgd_lr_poly_decay", "odsgd_fused_update_mult_static", "odsgd_get_iteration", "odsgd_set_iteration",
+    "odsgd_bind_grads", "odsgd_unbind_grads", "odsgd_global_update_bound", "odsgd_fused_update_bound",
+    "odsgd_ssgd_step_bound", "odsgd_step_bound", "odsgd_worker_local_update", "odsgd_shard_range",
 )
 
 
@@ -105,6 +109,15 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_get_iteration": ([vp, u64p], ci),
         "odsgd_set_iteration": ([vp, ctypes.c_uint64], ci),
         "odsgd_fused_update_mult_static": ([vp, pvp, ci, ctypes.POINTER(cf), ctypes.POINTER(cf), vp], ci),
+        "odsgd_bind_grads": ([vp, pvp, ctypes.POINTER(ci)], ci),
+        "odsgd_unbind_grads": ([vp, ci], ci),
+        "odsgd_global_update_bound": ([vp, ci, vp], ci),
+        "odsgd_fused_update_bound": ([vp, ci, ci, vp], ci),
+        "odsgd_ssgd_step_bound": ([vp, ci, vp], ci),
+        "odsgd_step_bound": ([vp, ci, vp], ci),
+        "odsgd_worker_local_update": ([vp, ci, vp, vp, ci, vp], ci),
+        "odsgd_shard_range": ([ctypes.c_size_t, ci, ci, ctypes.POINTER(ctypes.c_size_t),
+                               ctypes.POINTER(ctypes.c_size_t)], ci),
     }
     for name, (argtypes, restype) in sig.items():
         fn = getattr(lib, name)  # AttributeError if the library lacks a declared symbol
@@ -155,10 +168,29 @@ class GradTable:
         return iter(self.tensors)
 
 
+class BoundGrads:
+    """A gradient table the library has checked once (odsgd_bind_grads): passing it to the update
+    calls skips the per-call validation.  Keeps the tensors alive; `unbind()` frees the slot."""
+
+    def __init__(self, ctx: "Odsgd", grads: Sequence[torch.Tensor], slot: int):
+        self.ctx, self.tensors, self.slot = ctx, list(grads), slot
+
+    def unbind(self) -> None:
+        if self.slot >= 0:
+            self.ctx._check(self.ctx._lib.odsgd_unbind_grads(self.ctx._h, self.slot))
+            self.slot = -1
+
+    def __len__(self) -> int:
+        return len(self.tensors)
+
+    def __iter__(self):
+        return iter(self.tensors)
+
+
 class Odsgd:
     """One context of the CUDA library (see include/odsgd.h for the semantics of each call)."""
 
-    def __init__(self, w_a: torch.Tensor, v: torch.Tensor, *, n_workers: int, lr: float, local_lr: float,
+    def __init__(self, w_a: torch.Tensor, v: Optional[torch.Tensor], *, n_workers: int, lr: float, local_lr: float,
                  momentum: float, wd: float, w_b: Optional[torch.Tensor] = None,
                  w_delayed: Optional[torch.Tensor] = None,
                  local: Optional[Sequence[Optional[torch.Tensor]]] = None,
@@ -219,6 +251,18 @@ class Odsgd:
         cost of a step on small parameter sets)."""
         return GradTable(grads, self.n_workers, self.n_params)
 
+    def bind_grads(self, grads: Sequence[torch.Tensor]) -> "BoundGrads":
+        """odsgd_bind_grads: the library validates the table once; global_update / fused_update /
+        ssgd_step / step_update then take the returned object in place of the tensor list."""
+        slot = ctypes.c_int(-1)
+        self._check(self._lib.odsgd_bind_grads(self._h, self._grad_table(grads), ctypes.byref(slot)))
+        return BoundGrads(self, grads, slot.value)
+
+    def _slot(self, grads: "BoundGrads") -> int:
+        if grads.ctx is not self or grads.slot < 0:
+            raise ValueError("gradient table is bound to another context, or was unbound")
+        return grads.slot
+
     def close(self) -> None:
         if self._h:
             self._lib.odsgd_destroy(self._h)
@@ -232,7 +276,10 @@ class Odsgd:
 
     # -- the update calls
     def global_update(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
-        self._check(self._lib.odsgd_global_update(self._h, self._grad_table(grads), _stream_handle(stream)))
+        if isinstance(grads, BoundGrads):
+            self._check(self._lib.odsgd_global_update_bound(self._h, self._slot(grads), _stream_handle(stream)))
+        else:
+            self._check(self._lib.odsgd_global_update(self._h, self._grad_table(grads), _stream_handle(stream)))
         self._bound = grads
 
     def local_update(self, worker_id: int, stream: Optional[torch.cuda.Stream] = None) -> None:
@@ -240,9 +287,29 @@ class Odsgd:
 
     def fused_update(self, grads: Sequence[torch.Tensor], worker_id: int,
                      stream: Optional[torch.cuda.Stream] = None) -> None:
-        self._check(self._lib.odsgd_fused_update(self._h, self._grad_table(grads), worker_id,
-                                                 _stream_handle(stream)))
+        if isinstance(grads, BoundGrads):
+            self._check(self._lib.odsgd_fused_update_bound(self._h, self._slot(grads), worker_id,
+                                                           _stream_handle(stream)))
+        else:
+            self._check(self._lib.odsgd_fused_update(self._h, self._grad_table(grads), worker_id,
+                                                     _stream_handle(stream)))
         self._bound = grads
+
+    def fused_update_bound_raw(self, slot: int, worker_id: int, stream_handle: int) -> int:
+        """odsgd_fused_update_bound with nothing around it: slot index and raw stream handle in,
+        error code out (check it with `check`).  For loops where the marshalling of the regular
+        wrapper is comparable to the kernel itself."""
+        return self._lib.odsgd_fused_update_bound(self._h, slot, worker_id, stream_handle)
+
+    def check(self, rc: int) -> None:
+        self._check(rc)
+
+    def worker_local_update(self, worker_id: int, w_bak: torch.Tensor, grad: torch.Tensor, no_delay: bool = False,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+        """odsgd_worker_local_update: local[worker_id] = LocalRule(w_bak, grad) on explicit inputs."""
+        self._check(self._lib.odsgd_worker_local_update(self._h, worker_id, _dev_ptr(w_bak, "w_bak", self.n_params),
+                                                        _dev_ptr(grad, "grad", self.n_params), int(bool(no_delay)),
+                                                        _stream_handle(stream)))
 
     def fused_update_host(self, host_grads: Sequence[torch.Tensor], dev_staging: Sequence[torch.Tensor],
                           worker_id: int, host_local_out: Optional[torch.Tensor] = None,
@@ -267,7 +334,10 @@ class Odsgd:
         self._bound = list(dev_staging)
 
     def ssgd_step(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
-        self._check(self._lib.odsgd_ssgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
+        if isinstance(grads, BoundGrads):
+            self._check(self._lib.odsgd_ssgd_step_bound(self._h, self._slot(grads), _stream_handle(stream)))
+        else:
+            self._check(self._lib.odsgd_ssgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
 
     def asgd_step(self, worker_id: int, grad: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
         self._check(self._lib.odsgd_asgd_step(self._h, worker_id, _dev_ptr(grad, "grad", self.n_params),
@@ -279,7 +349,10 @@ class Odsgd:
 
     def step_update(self, grads: Sequence[torch.Tensor], stream: Optional[torch.cuda.Stream] = None) -> None:
         """odsgd_step: one iteration of Algorithm 2's state machine (warm-up SSGD, then OD-SGD)."""
-        self._check(self._lib.odsgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
+        if isinstance(grads, BoundGrads):
+            self._check(self._lib.odsgd_step_bound(self._h, self._slot(grads), _stream_handle(stream)))
+        else:
+            self._check(self._lib.odsgd_step(self._h, self._grad_table(grads), _stream_handle(stream)))
         self._bound = grads
 
     def set_warmup(self, wp: int) -> None:
@@ -394,6 +467,15 @@ class Odsgd:
 
 def version() -> int:
     return load_library().odsgd_version()
+
+
+def shard_range(n_params: int, n_ranks: int, rank: int) -> tuple:
+    """odsgd_shard_range: the slice [begin, end) of the arena that rank `rank` of `n_ranks` owns."""
+    b, e = ctypes.c_size_t(), ctypes.c_size_t()
+    rc = load_library().odsgd_shard_range(n_params, n_ranks, rank, ctypes.byref(b), ctypes.byref(e))
+    if rc != OK:
+        raise OdsgdError(rc, "odsgd_shard_range: n_ranks >= 1 and 0 <= rank < n_ranks are required")
+    return b.value, e.value
 
 
 # The C entry points under their own names, for callers that prefer the flat C style.

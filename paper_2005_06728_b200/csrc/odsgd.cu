@@ -1,12 +1,15 @@
 // Host side of the OD-SGD update library: context, validation, kernel selection
 // and launches behind the C ABI declared in odsgd.h.  No torch types, no
-// allocation of parameter-sized memory, no synchronisation.
+// allocation of parameter-sized memory, no synchronisation.  The per-call path of the
+// update entry points allocates nothing on the host either: buffers are enumerated into
+// fixed arrays on the stack and error texts are only built when a call fails.
 #include <cuda_runtime.h>
 
 #include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -23,11 +26,12 @@ struct odsgd_ctx {
     int cur = 0;  // index of the half that holds the current weights
     bool pingpong = false;
     float* w_delayed = nullptr;  // in-place layout: optional backup arena
-    float* v = nullptr;
+    float* v = nullptr;          // NULL only in a worker-only context
     float* local[ODSGD_MAX_WORKERS] = {};
     float* mean_square[ODSGD_MAX_WORKERS] = {};
     size_t n = 0;
     std::vector<size_t> offsets;
+    bool offsets_vec_ok = true;  // every tensor offset is a multiple of 4 elements
     int n_workers = 0;
     float lr = 0, local_lr = 0, momentum = 0, wd = 0;
     uint32_t flags = 0;
@@ -50,7 +54,17 @@ struct odsgd_ctx {
     // host-buffer entry point with a separate copy stream: ordering between the two streams
     cudaEvent_t ev_kernel_done = nullptr;  // recorded on the compute stream after the update kernel
     cudaEvent_t ev_copy_done = nullptr;    // recorded on the copy stream after the device-to-host copy
-    bool copy_pending = false;
+    bool copy_pending = false;             // ev_copy_done guards a copy-back no later kernel may overtake
+    bool copy_waited = false;              // a stream has been made to wait for that copy already ...
+    cudaStream_t copy_waited_on = nullptr; // ... this one: work enqueued on it later is ordered behind the copy
+    // gradient tables checked once by odsgd_bind_grads
+    struct Binding {
+        bool used = false;
+        uint64_t epoch = 0;  // state_epoch at the time the table was checked
+        const float* g[ODSGD_MAX_WORKERS] = {};
+    };
+    Binding bindings[ODSGD_MAX_BINDINGS];
+    uint64_t state_epoch = 0;  // bumped whenever the set of state buffers changes
     // resident CTAs per SM by (kernel, block size); 0 = that block size cannot be launched
     std::map<std::pair<const void*, int>, int> occupancy;
     std::string err;
@@ -59,7 +73,6 @@ struct odsgd_ctx {
 namespace {
 
 thread_local std::string g_create_err;
-
 
 int fail(odsgd_ctx* ctx, int code, const std::string& msg) {
     if (ctx) ctx->err = msg; else g_create_err = msg;
@@ -85,47 +98,72 @@ std::string label(const Named& b) {
     return buf;
 }
 
-// State buffers of a context, for alias checks.
-std::vector<Named> state_buffers(const odsgd_ctx* c) {
-    std::vector<Named> s;
-    s.push_back({c->w[0], "w_a", -1});
-    if (c->w[1]) s.push_back({c->w[1], "w_b", -1});
-    if (c->w_delayed) s.push_back({c->w_delayed, "w_delayed", -1});
-    s.push_back({c->v, "v", -1});
-    for (int m = 0; m < c->n_workers; ++m) {
-        if (c->local[m]) s.push_back({c->local[m], "local", m});
-        if (c->mean_square[m]) s.push_back({c->mean_square[m], "mean_square", m});
+// A short list of named buffers on the stack (no heap traffic on the per-call path).
+template <int CAP>
+struct BufList {
+    Named b[CAP];
+    int n = 0;
+    void add(const void* p, const char* name, int idx) {
+        if (n < CAP) b[n++] = Named{p, name, idx};
     }
-    if (c->server_ms) s.push_back({c->server_ms, "server_mean_square", -1});
-    return s;
+};
+constexpr int kMaxState = 5 + 2 * ODSGD_MAX_WORKERS;
+using StateList = BufList<kMaxState>;
+using CallList = BufList<kMaxState + ODSGD_MAX_WORKERS + 4>;
+
+// State buffers of a context, for alias checks.
+void state_buffers(const odsgd_ctx* c, StateList* s) {
+    s->n = 0;
+    s->add(c->w[0], "w_a", -1);
+    if (c->w[1]) s->add(c->w[1], "w_b", -1);
+    if (c->w_delayed) s->add(c->w_delayed, "w_delayed", -1);
+    if (c->v) s->add(c->v, "v", -1);
+    for (int m = 0; m < c->n_workers; ++m) {
+        if (c->local[m]) s->add(c->local[m], "local", m);
+        if (c->mean_square[m]) s->add(c->mean_square[m], "mean_square", m);
+    }
+    if (c->server_ms) s->add(c->server_ms, "server_mean_square", -1);
 }
 
-int check_distinct(odsgd_ctx* err_ctx, const std::vector<Named>& s, size_t bytes) {
-    for (size_t i = 0; i < s.size(); ++i)
-        for (size_t j = i + 1; j < s.size(); ++j)
-            if (overlap(s[i].p, s[j].p, bytes))
-                return fail(err_ctx, ODSGD_ERR_OVERLAP, label(s[i]) + " overlaps " + label(s[j]));
+int check_distinct(odsgd_ctx* err_ctx, const StateList& s, size_t bytes) {
+    for (int i = 0; i < s.n; ++i)
+        for (int j = i + 1; j < s.n; ++j)
+            if (overlap(s.b[i].p, s.b[j].p, bytes))
+                return fail(err_ctx, ODSGD_ERR_OVERLAP, label(s.b[i]) + " overlaps " + label(s.b[j]));
     return ODSGD_OK;
 }
 
-// Vector width usable for a call: 4 lanes when every pointer is 16-byte aligned, else
-// 1 lane if the context allows it.  Returns 0 and sets the error otherwise.
-int lanes_for(odsgd_ctx* c, const std::vector<Named>& ptrs) {
-    bool all16 = true;
-    for (const Named& b : ptrs) {
+// One outside buffer (a gradient, a caller-supplied backup) against the context's state.
+int check_outside(odsgd_ctx* c, const StateList& st, const Named& g) {
+    const size_t bytes = c->n * sizeof(float);
+    for (int i = 0; i < st.n; ++i)
+        if (overlap(g.p, st.b[i].p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, label(g) + " overlaps " + label(st.b[i]));
+    return ODSGD_OK;
+}
+
+// Vector width usable for a call: 4 lanes when every pointer it touches is 16-byte aligned,
+// else 1 lane if the context allows it.  Returns 0 and sets the error otherwise.  The common
+// case is decided from the OR of all addresses; the buffers are only walked by name to word
+// the error.
+template <int CAP>
+int lanes_for(odsgd_ctx* c, const BufList<CAP>& ptrs) {
+    uintptr_t bits = 0;
+    for (int i = 0; i < ptrs.n; ++i) bits |= reinterpret_cast<uintptr_t>(ptrs.b[i].p);
+    if ((bits & 15) == 0) return 4;
+    const bool scalar_ok = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) != 0;
+    if ((bits & 3) == 0 && scalar_ok) return 1;
+    for (int i = 0; i < ptrs.n; ++i) {
+        const Named& b = ptrs.b[i];
         if (!aligned(b.p, 4)) {
             fail(c, ODSGD_ERR_ALIGN, label(b) + " is not 4-byte aligned");
             return 0;
         }
-        if (!aligned(b.p, 16)) {
-            if (!(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED)) {
-                fail(c, ODSGD_ERR_ALIGN, label(b) + " is not 16-byte aligned (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
-                return 0;
-            }
-            all16 = false;
+        if (!aligned(b.p, 16) && !scalar_ok) {
+            fail(c, ODSGD_ERR_ALIGN, label(b) + " is not 16-byte aligned (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
+            return 0;
         }
     }
-    return all16 ? 4 : 1;
+    return 1;
 }
 
 int grid_for(const odsgd_ctx* c, unsigned long long n, int lanes, int block, int per_thread, int resident_default) {
@@ -182,56 +220,62 @@ int too_wide(odsgd_ctx* c, int block) {
     return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
 }
 
+// `dry`: stop after the checks that can still refuse the launch (block size against the
+// kernel's register use), so that a caller can validate everything before it enqueues copies.
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
-int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
     auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT, BB, UB>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    const int grid = grid_for(c, a.n, NL, block, UB, kServerCtasPerSm);
+    if (dry) return ODSGD_OK;
+    const int grid = grid_for(c, a.n, NL, block, server_vectors_per_thread(LOCAL, RULE, UB), kServerCtasPerSm);
     kernel<<<grid, block, 0, st>>>(a);
     return after_launch(c, "server kernel launch");
 }
 
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
-int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
+int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry) {
     // few workers: the pass is close to a copy and wants the shallow, wide shape
     if constexpr (LOCAL != kLocalAll) {
         if (a.n_workers <= kFewWorkers)
-            return launch_server_k<DET, NL, LOCAL, RULE, MULT, kFewBatch, kFewUnroll>(c, a, st);
+            return launch_server_k<DET, NL, LOCAL, RULE, MULT, kFewBatch, kFewUnroll>(c, a, st, dry);
     }
-    return launch_server_k<DET, NL, LOCAL, RULE, MULT, kBatch, kUnroll>(c, a, st);
+    return launch_server_k<DET, NL, LOCAL, RULE, MULT, kBatch, kUnroll>(c, a, st, dry);
 }
 
 template <bool DET, int NL, int LOCAL, int RULE>
-int launch_server_t(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
-    return c->mult_on ? launch_server_m<DET, NL, LOCAL, RULE, true>(c, a, st)
-                      : launch_server_m<DET, NL, LOCAL, RULE, false>(c, a, st);
+int launch_server_t(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t st, bool dry) {
+    return mult ? launch_server_m<DET, NL, LOCAL, RULE, true>(c, a, st, dry)
+                : launch_server_m<DET, NL, LOCAL, RULE, false>(c, a, st, dry);
 }
 
 template <bool DET, int NL, int LOCAL>
-int launch_server_r(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st) {
-    if (LOCAL == kLocalNone) return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, st);
+int launch_server_r(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t st, bool dry) {
+    if (LOCAL == kLocalNone) return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
     switch (c->local_rule) {
-        case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, st);
-        case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, st);
-        case ODSGD_LOCAL_MOMENTUM: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_MOMENTUM>(c, a, st);
-        default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, st);
+        case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
+        case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, mult, st, dry);
+        case ODSGD_LOCAL_MOMENTUM: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_MOMENTUM>(c, a, mult, st, dry);
+        default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, mult, st, dry);
     }
 }
 
 template <bool DET, int NL>
-int launch_server_l(odsgd_ctx* c, const ServerArgs& a, int local_mode, cudaStream_t st) {
+int launch_server_l(odsgd_ctx* c, const ServerArgs& a, int local_mode, bool mult, cudaStream_t st, bool dry) {
     switch (local_mode) {
-        case kLocalNone: return launch_server_r<DET, NL, kLocalNone>(c, a, st);
-        case kLocalOne: return launch_server_r<DET, NL, kLocalOne>(c, a, st);
-        default: return launch_server_r<DET, NL, kLocalAll>(c, a, st);
+        case kLocalNone: return launch_server_r<DET, NL, kLocalNone>(c, a, mult, st, dry);
+        case kLocalOne: return launch_server_r<DET, NL, kLocalOne>(c, a, mult, st, dry);
+        default: return launch_server_r<DET, NL, kLocalAll>(c, a, mult, st, dry);
     }
 }
 
-int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, cudaStream_t st) {
+int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, bool mult, cudaStream_t st, bool dry) {
     const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
-    if (det) return lanes == 4 ? launch_server_l<true, 4>(c, a, local_mode, st) : launch_server_l<true, 1>(c, a, local_mode, st);
-    return lanes == 4 ? launch_server_l<false, 4>(c, a, local_mode, st) : launch_server_l<false, 1>(c, a, local_mode, st);
+    if (det)
+        return lanes == 4 ? launch_server_l<true, 4>(c, a, local_mode, mult, st, dry)
+                          : launch_server_l<true, 1>(c, a, local_mode, mult, st, dry);
+    return lanes == 4 ? launch_server_l<false, 4>(c, a, local_mode, mult, st, dry)
+                      : launch_server_l<false, 1>(c, a, local_mode, mult, st, dry);
 }
 
 template <bool DET, int NL, int RULE, bool SERVER>
@@ -289,36 +333,50 @@ LocalParams local_params(const odsgd_ctx* c) {
     return p;
 }
 
-// Run before every kernel launch: the context's device must be current, and a copy-back of
-// local weights that odsgd_fused_update_host put on a separate copy stream must be out before
-// a later kernel overwrites a local arena (`st` is made to wait for it).
+// Run before every kernel that may write a local arena: the context's device must be
+// current, and a copy-back of local weights that odsgd_fused_update_host put on a separate
+// copy stream must be out before the kernel overwrites that arena.  Every stream that comes
+// by is made to wait for the copy (work behind it on the same stream is ordered anyway); the
+// guard stays up until a later host-buffer call records a newer copy.
 int before_launch(odsgd_ctx* c, cudaStream_t st) {
     const int rc_dev = on_own_device(c);
     if (rc_dev != ODSGD_OK) return rc_dev;
     if (!c->copy_pending) return ODSGD_OK;
+    if (c->copy_waited && c->copy_waited_on == st) return ODSGD_OK;
     const cudaError_t e = cudaStreamWaitEvent(st, c->ev_copy_done, 0);
     if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("stream wait: ") + cudaGetErrorString(e));
-    c->copy_pending = false;
+    c->copy_waited = true;
+    c->copy_waited_on = st;
     return ODSGD_OK;
 }
 
 // Checks a table of gradient pointers against the context's state buffers.
-int check_grads(odsgd_ctx* c, const float* const* grads, std::vector<Named>* ptrs) {
+int check_grads(odsgd_ctx* c, const float* const* grads) {
     if (!grads) return fail(c, ODSGD_ERR_ARG, "worker_grads is NULL");
-    const size_t bytes = c->n * sizeof(float);
-    const std::vector<Named> st = state_buffers(c);
+    StateList st;
+    state_buffers(c, &st);
     for (int m = 0; m < c->n_workers; ++m) {
         if (!grads[m]) return fail(c, ODSGD_ERR_ARG, "worker_grads[" + std::to_string(m) + "] is NULL");
-        const Named g{grads[m], "worker_grads", m};
-        for (const Named& s : st)
-            if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, label(g) + " overlaps " + label(s));
-        ptrs->push_back(g);
+        const int rc = check_outside(c, st, Named{grads[m], "worker_grads", m});
+        if (rc != ODSGD_OK) return rc;
     }
     return ODSGD_OK;
 }
 
+// A fully validated server-kernel launch: arguments, vector width, and what the context's
+// state becomes once the launch is in the stream.
+struct ServerPlan {
+    ServerArgs a;
+    int lanes = 0;
+    int local_mode = kLocalNone;
+    bool mult = false;
+    bool keep_backup = false;
+    int next_cur = 0;
+    const float* delayed_after = nullptr;
+};
+
 // Local mode and outputs for a fused call; fills a.x / a.ms / a.local_worker.
-int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mode, std::vector<Named>* ptrs) {
+int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mode, CallList* ptrs) {
     if (worker_id >= c->n_workers || worker_id < -1) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
     const bool need_ms = needs_state(c->local_rule);
     if (worker_id >= 0) {
@@ -327,8 +385,8 @@ int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mo
         a->x[0] = c->local[worker_id];
         a->ms[0] = c->mean_square[worker_id];
         a->local_worker = worker_id;
-        ptrs->push_back({a->x[0], "local", worker_id});
-        if (need_ms) ptrs->push_back({a->ms[0], "mean_square", worker_id});
+        ptrs->add(a->x[0], "local", worker_id);
+        if (need_ms) ptrs->add(a->ms[0], "mean_square", worker_id);
         *local_mode = kLocalOne;
         return ODSGD_OK;
     }
@@ -338,8 +396,8 @@ int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mo
         a->ms[m] = c->mean_square[m];
         if (c->local[m]) {
             if (need_ms && !c->mean_square[m]) return fail(c, ODSGD_ERR_STATE, "no mean-square arena for worker " + std::to_string(m));
-            ptrs->push_back({a->x[m], "local", m});
-            if (need_ms) ptrs->push_back({a->ms[m], "mean_square", m});
+            ptrs->add(a->x[m], "local", m);
+            if (need_ms) ptrs->add(a->ms[m], "mean_square", m);
             ++count;
         }
     }
@@ -348,19 +406,21 @@ int bind_local_outputs(odsgd_ctx* c, int worker_id, ServerArgs* a, int* local_mo
     return ODSGD_OK;
 }
 
-// Shared body of the global, fused and SSGD calls.
-//   keep_backup: OD-SGD server step (the old weights stay available to the workers)
-//   local_id:    -2 none, -1 all workers, >= 0 one worker
-int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, void* stream,
-                bool first_delayed_step = false) {
-    if (!c) return ODSGD_ERR_ARG;
-    std::vector<Named> ptrs;
-    int rc = check_grads(c, grads, &ptrs);
-    if (rc != ODSGD_OK) return rc;
-
-    ServerArgs a;
+// Builds the plan of a global, fused or SSGD call from a gradient table that has already been
+// checked against the state buffers (check_grads, at call or at bind time).
+//   keep_backup:  OD-SGD server step (the old weights stay available to the workers)
+//   local_id:     -2 none, -1 all workers, >= 0 one worker
+//   static_table: device address of a multiplier table to use instead of the context's own
+int plan_server(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, bool first_delayed_step,
+                const unsigned char* static_table, ServerPlan* p) {
+    if (!c->v) return fail(c, ODSGD_ERR_STATE, "a worker-only context (ODSGD_FLAG_WORKER_ONLY) has no server state");
+    ServerArgs& a = p->a;
     memset(&a, 0, sizeof a);
-    for (int m = 0; m < c->n_workers; ++m) a.g[m] = grads[m];
+    CallList ptrs;
+    for (int m = 0; m < c->n_workers; ++m) {
+        a.g[m] = grads[m];
+        ptrs.add(grads[m], "worker_grads", m);
+    }
     a.v = c->v;
     a.n = c->n;
     a.n_workers = c->n_workers;
@@ -370,59 +430,104 @@ int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
     a.wd = c->wd;
     a.lp = local_params(c);
     a.lp.first = first_delayed_step ? 1 : 0;
-    if (c->mult_on) {
+    p->mult = static_table != nullptr || c->mult_on;
+    if (p->mult) {
         const size_t nt = c->offsets.size() - 1;
-        unsigned char* base = static_cast<unsigned char*>(c->table_dev);
+        const unsigned char* base = static_table ? static_table : static_cast<const unsigned char*>(c->table_dev);
         a.t_off = reinterpret_cast<const unsigned long long*>(base);
         a.t_lr_mult = reinterpret_cast<const float*>(base + (nt + 1) * sizeof(unsigned long long));
         a.t_wd_mult = a.t_lr_mult + nt;
         a.n_tensors = (unsigned int)nt;
     }
     a.w_in = c->w[c->cur];
-    const float* delayed_after = nullptr;
-    int next_cur = c->cur;
+    p->keep_backup = keep_backup;
+    p->delayed_after = nullptr;
+    p->next_cur = c->cur;
     if (keep_backup && c->pingpong) {
         a.w_out = c->w[c->cur ^ 1];
-        delayed_after = c->w[c->cur];
-        next_cur = c->cur ^ 1;
+        p->delayed_after = c->w[c->cur];
+        p->next_cur = c->cur ^ 1;
     } else {
         a.w_out = c->w[c->cur];
         if (keep_backup && c->w_delayed) {
             a.w_prev = c->w_delayed;
-            delayed_after = c->w_delayed;
+            p->delayed_after = c->w_delayed;
         }
     }
-    ptrs.push_back({a.w_in, "w", -1});
-    ptrs.push_back({a.w_out, "w", -1});
-    ptrs.push_back({a.v, "v", -1});
-    if (a.w_prev) ptrs.push_back({a.w_prev, "w_delayed", -1});
+    ptrs.add(a.w_in, "w", -1);
+    ptrs.add(a.w_out, "w", -1);
+    ptrs.add(a.v, "v", -1);
+    if (a.w_prev) ptrs.add(a.w_prev, "w_delayed", -1);
 
-    int local_mode = kLocalNone;
+    p->local_mode = kLocalNone;
     if (local_id >= -1) {
-        rc = bind_local_outputs(c, local_id, &a, &local_mode, &ptrs);
+        const int rc = bind_local_outputs(c, local_id, &a, &p->local_mode, &ptrs);
         if (rc != ODSGD_OK) return rc;
     }
-    int lanes = lanes_for(c, ptrs);
-    if (lanes == 0) return ODSGD_ERR_ALIGN;
-    if (c->mult_on && lanes == 4) {
-        // a 128-bit vector must not straddle two tensors (set_tensor_multipliers has checked that
-        // the scalar path is allowed when it would)
-        for (size_t o : c->offsets)
-            if (o % 4 != 0) { lanes = 1; break; }
-    }
-
-    rc = before_launch(c, static_cast<cudaStream_t>(stream));
-    if (rc != ODSGD_OK) return rc;
-    rc = launch_server(c, a, lanes, local_mode, static_cast<cudaStream_t>(stream));
-    if (rc != ODSGD_OK) return rc;
-
-    c->cur = next_cur;
-    c->step += 1;
-    c->delayed = delayed_after;
-    c->grads_bound = keep_backup;
-    if (keep_backup)
-        for (int m = 0; m < c->n_workers; ++m) c->bound[m] = grads[m];
+    p->lanes = lanes_for(c, ptrs);
+    if (p->lanes == 0) return ODSGD_ERR_ALIGN;
+    // with multipliers a 128-bit vector must not straddle two tensors (the calls that switch
+    // them on have checked that the scalar path is allowed when it would)
+    if (p->mult && p->lanes == 4 && !c->offsets_vec_ok) p->lanes = 1;
     return ODSGD_OK;
+}
+
+// Launches a plan (or, with dry = true, only runs the checks that could still refuse it)
+// and moves the context's state on.
+int run_server(odsgd_ctx* c, const ServerPlan& p, cudaStream_t st, bool dry) {
+    int rc = dry ? on_own_device(c) : before_launch(c, st);
+    if (rc != ODSGD_OK) return rc;
+    rc = launch_server(c, p.a, p.lanes, p.local_mode, p.mult, st, dry);
+    if (rc != ODSGD_OK || dry) return rc;
+    c->cur = p.next_cur;
+    c->step += 1;
+    c->delayed = p.delayed_after;
+    c->grads_bound = p.keep_backup;
+    if (p.keep_backup)
+        for (int m = 0; m < c->n_workers; ++m) c->bound[m] = p.a.g[m];
+    return ODSGD_OK;
+}
+
+// Shared body of the global, fused and SSGD calls on an unchecked gradient table.
+int server_call(odsgd_ctx* c, const float* const* grads, bool keep_backup, int local_id, void* stream,
+                bool first_delayed_step = false) {
+    if (!c) return ODSGD_ERR_ARG;
+    int rc = check_grads(c, grads);
+    if (rc != ODSGD_OK) return rc;
+    ServerPlan p;
+    rc = plan_server(c, grads, keep_backup, local_id, first_delayed_step, nullptr, &p);
+    if (rc != ODSGD_OK) return rc;
+    return run_server(c, p, static_cast<cudaStream_t>(stream), false);
+}
+
+// The same on a table odsgd_bind_grads has checked: no scan of the state buffers.
+int bound_call(odsgd_ctx* c, int slot, bool keep_backup, int local_id, void* stream, bool first_delayed_step = false) {
+    if (!c) return ODSGD_ERR_ARG;
+    if (slot < 0 || slot >= ODSGD_MAX_BINDINGS || !c->bindings[slot].used)
+        return fail(c, ODSGD_ERR_ARG, "no gradient table is bound to slot " + std::to_string(slot));
+    const odsgd_ctx::Binding& b = c->bindings[slot];
+    if (b.epoch != c->state_epoch)
+        return fail(c, ODSGD_ERR_STATE, "the context's buffers changed after slot " + std::to_string(slot) +
+                                            " was bound: bind the gradient table again");
+    ServerPlan p;
+    const int rc = plan_server(c, b.g, keep_backup, local_id, first_delayed_step, nullptr, &p);
+    if (rc != ODSGD_OK) return rc;
+    return run_server(c, p, static_cast<cudaStream_t>(stream), false);
+}
+
+// Algorithm 2's schedule: which server call iteration c->iter is.
+template <typename F>
+int scheduled_step(odsgd_ctx* c, F call) {
+    int rc;
+    if (c->iter < c->wp) {
+        rc = call(false, -2, false);  // warm-up stage: SSGD
+    } else {
+        // from the last warm-up iteration on: server step + local update of every worker; at
+        // iteration wp itself the gradients were taken on the global weights (no delay yet)
+        rc = call(true, -1, c->iter == c->wp);
+    }
+    if (rc == ODSGD_OK) c->iter += 1;
+    return rc;
 }
 
 }  // namespace
@@ -448,7 +553,10 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
     if (!out) return fail(nullptr, ODSGD_ERR_ARG, "out is NULL");
     *out = nullptr;
     if (!d) return fail(nullptr, ODSGD_ERR_ARG, "desc is NULL");
-    if (!d->w_a || !d->v) return fail(nullptr, ODSGD_ERR_ARG, "w_a and v must not be NULL");
+    constexpr uint32_t known =
+        ODSGD_FLAG_DETERMINISTIC | ODSGD_FLAG_ALLOW_UNALIGNED | ODSGD_FLAG_ALLOW_FMA | ODSGD_FLAG_WORKER_ONLY;
+    const bool worker_only = (d->flags & ODSGD_FLAG_WORKER_ONLY) != 0;
+    if (!d->w_a || (!d->v && !worker_only)) return fail(nullptr, ODSGD_ERR_ARG, "w_a and v must not be NULL");
     if (d->n_params == 0) return fail(nullptr, ODSGD_ERR_ARG, "n_params is 0");
     if (d->n_workers < 1 || d->n_workers > ODSGD_MAX_WORKERS)
         return fail(nullptr, ODSGD_ERR_ARG, "n_workers must be in 1.." + std::to_string(ODSGD_MAX_WORKERS));
@@ -459,8 +567,7 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
     for (size_t t = 0; t < d->n_tensors; ++t)
         if (d->tensor_offsets[t + 1] <= d->tensor_offsets[t])
             return fail(nullptr, ODSGD_ERR_ARG, "tensor_offsets must be strictly ascending (at tensor " + std::to_string(t) + ")");
-    if (d->flags & ~(ODSGD_FLAG_DETERMINISTIC | ODSGD_FLAG_ALLOW_UNALIGNED | ODSGD_FLAG_ALLOW_FMA))
-        return fail(nullptr, ODSGD_ERR_ARG, "unknown flag bits");
+    if (d->flags & ~known) return fail(nullptr, ODSGD_ERR_ARG, "unknown flag bits");
     if ((d->flags & ODSGD_FLAG_DETERMINISTIC) && (d->flags & ODSGD_FLAG_ALLOW_FMA))
         return fail(nullptr, ODSGD_ERR_ARG, "ODSGD_FLAG_DETERMINISTIC and ODSGD_FLAG_ALLOW_FMA exclude each other");
 
@@ -474,6 +581,8 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
     c->n = d->n_params;
     c->n_workers = d->n_workers;
     c->offsets.assign(d->tensor_offsets, d->tensor_offsets + d->n_tensors + 1);
+    for (size_t o : c->offsets)
+        if (o % 4 != 0) c->offsets_vec_ok = false;
     c->lr = d->lr;
     c->local_lr = d->local_lr;
     c->momentum = d->momentum;
@@ -482,11 +591,12 @@ int odsgd_create(odsgd_ctx** out, const odsgd_desc* d) {
     if (d->local)
         for (int m = 0; m < d->n_workers; ++m) c->local[m] = d->local[m];
 
-    const std::vector<Named> st = state_buffers(c);
+    StateList st;
+    state_buffers(c, &st);
     const size_t need = (d->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
-    for (const Named& b : st) {
-        if (!aligned(b.p, need)) {
-            const std::string msg = label(b) + " is not " + std::to_string(need) + "-byte aligned";
+    for (int i = 0; i < st.n; ++i) {
+        if (!aligned(st.b[i].p, need)) {
+            const std::string msg = label(st.b[i]) + " is not " + std::to_string(need) + "-byte aligned";
             delete c;
             return fail(nullptr, ODSGD_ERR_ALIGN, msg);
         }
@@ -531,6 +641,48 @@ int odsgd_ssgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stre
     return server_call(ctx, worker_grads, false, -2, stream);
 }
 
+int odsgd_bind_grads(odsgd_ctx* ctx, const float* const* worker_grads, int* slot) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (!slot) return fail(c, ODSGD_ERR_ARG, "slot is NULL");
+    *slot = -1;
+    int rc = check_grads(c, worker_grads);
+    if (rc != ODSGD_OK) return rc;
+    // alignment is a property of the table too: refuse now what every later call would refuse
+    CallList ptrs;
+    for (int m = 0; m < c->n_workers; ++m) ptrs.add(worker_grads[m], "worker_grads", m);
+    if (lanes_for(c, ptrs) == 0) return ODSGD_ERR_ALIGN;
+    for (int s = 0; s < ODSGD_MAX_BINDINGS; ++s) {
+        odsgd_ctx::Binding& b = c->bindings[s];
+        if (b.used) continue;
+        b.used = true;
+        b.epoch = c->state_epoch;
+        for (int m = 0; m < ODSGD_MAX_WORKERS; ++m) b.g[m] = m < c->n_workers ? worker_grads[m] : nullptr;
+        *slot = s;
+        return ODSGD_OK;
+    }
+    return fail(c, ODSGD_ERR_UNSUPPORTED,
+                "all " + std::to_string(ODSGD_MAX_BINDINGS) + " binding slots are in use (odsgd_unbind_grads frees one)");
+}
+
+int odsgd_unbind_grads(odsgd_ctx* ctx, int slot) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (slot < 0 || slot >= ODSGD_MAX_BINDINGS || !ctx->bindings[slot].used)
+        return fail(ctx, ODSGD_ERR_ARG, "no gradient table is bound to slot " + std::to_string(slot));
+    ctx->bindings[slot].used = false;
+    return ODSGD_OK;
+}
+
+int odsgd_global_update_bound(odsgd_ctx* ctx, int slot, void* stream) { return bound_call(ctx, slot, true, -2, stream); }
+
+int odsgd_fused_update_bound(odsgd_ctx* ctx, int slot, int worker_id, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    if (worker_id < -1 || worker_id >= ctx->n_workers) return fail(ctx, ODSGD_ERR_ARG, "worker_id out of range");
+    return bound_call(ctx, slot, true, worker_id, stream);
+}
+
+int odsgd_ssgd_step_bound(odsgd_ctx* ctx, int slot, void* stream) { return bound_call(ctx, slot, false, -2, stream); }
+
 int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     if (!ctx) return ODSGD_ERR_ARG;
     odsgd_ctx* c = ctx;
@@ -548,12 +700,56 @@ int odsgd_local_update(odsgd_ctx* ctx, int worker_id, void* stream) {
     a.w_out = nullptr;
     a.n = c->n;
     a.lp = local_params(c);
-    std::vector<Named> ptrs = {{a.w_bak, "w_delayed", -1}, {a.g, "worker_grads", worker_id}, {a.x, "local", worker_id}};
-    if (need_ms) ptrs.push_back({a.ms, "mean_square", worker_id});
+    BufList<4> ptrs;
+    ptrs.add(a.w_bak, "w_delayed", -1);
+    ptrs.add(a.g, "worker_grads", worker_id);
+    ptrs.add(a.x, "local", worker_id);
+    if (need_ms) ptrs.add(a.ms, "mean_square", worker_id);
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
     const int rc_copy = before_launch(c, static_cast<cudaStream_t>(stream));
     if (rc_copy != ODSGD_OK) return rc_copy;
+    return launch_local(c, a, lanes, false, static_cast<cudaStream_t>(stream));
+}
+
+int odsgd_worker_local_update(odsgd_ctx* ctx, int worker_id, const float* w_bak, const float* grad, int no_delay,
+                              void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
+    if (!w_bak || !grad) return fail(c, ODSGD_ERR_ARG, "w_bak / grad is NULL");
+    if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no local buffer for worker " + std::to_string(worker_id));
+    const bool need_ms = needs_state(c->local_rule);
+    if (need_ms && !c->mean_square[worker_id]) return fail(c, ODSGD_ERR_STATE, "no state arena (mean square / velocity) for that worker");
+    const size_t bytes = c->n * sizeof(float);
+    StateList st;
+    state_buffers(c, &st);
+    int rc = check_outside(c, st, Named{grad, "grad", -1});
+    if (rc != ODSGD_OK) return rc;
+    // the backup may be one of the context's own weight arenas (the replica the pull landed in),
+    // but not an arena this call writes
+    if (overlap(w_bak, c->local[worker_id], bytes))
+        return fail(c, ODSGD_ERR_OVERLAP, "w_bak overlaps local[" + std::to_string(worker_id) + "]");
+    if (need_ms && overlap(w_bak, c->mean_square[worker_id], bytes))
+        return fail(c, ODSGD_ERR_OVERLAP, "w_bak overlaps mean_square[" + std::to_string(worker_id) + "]");
+    LocalArgs a;
+    a.w_bak = w_bak;
+    a.g = grad;
+    a.x = c->local[worker_id];
+    a.ms = c->mean_square[worker_id];
+    a.w_out = nullptr;
+    a.n = c->n;
+    a.lp = local_params(c);
+    a.lp.first = no_delay ? 1 : 0;
+    BufList<4> ptrs;
+    ptrs.add(a.w_bak, "w_bak", -1);
+    ptrs.add(a.g, "grad", -1);
+    ptrs.add(a.x, "local", worker_id);
+    if (need_ms) ptrs.add(a.ms, "mean_square", worker_id);
+    const int lanes = lanes_for(c, ptrs);
+    if (lanes == 0) return ODSGD_ERR_ALIGN;
+    rc = before_launch(c, static_cast<cudaStream_t>(stream));
+    if (rc != ODSGD_OK) return rc;
     return launch_local(c, a, lanes, false, static_cast<cudaStream_t>(stream));
 }
 
@@ -566,16 +762,16 @@ int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, floa
     if (host_local_out && worker_id < 0) return fail(c, ODSGD_ERR_ARG, "host_local_out needs worker_id >= 0");
     for (int m = 0; m < c->n_workers; ++m)
         if (!host_grads[m] || !dev_staging[m]) return fail(c, ODSGD_ERR_ARG, "NULL entry in host_grads / dev_staging");
-    // validate before the first copy is enqueued
-    std::vector<Named> ptrs;
-    int rc = check_grads(c, dev_staging, &ptrs);
+    // everything that can refuse the update is checked before the first copy is enqueued, so a
+    // failed call leaves the staging arenas as they were
+    int rc = check_grads(c, dev_staging);
+    if (rc != ODSGD_OK) return rc;
+    ServerPlan p;
+    rc = plan_server(c, dev_staging, true, worker_id, false, nullptr, &p);
     if (rc != ODSGD_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t bytes = c->n * sizeof(float);
-    for (int m = 0; m < c->n_workers; ++m) {
-        const cudaError_t e = cudaMemcpyAsync(dev_staging[m], host_grads[m], bytes, cudaMemcpyHostToDevice, st);
-        if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("host-to-device copy: ") + cudaGetErrorString(e));
-    }
+    rc = run_server(c, p, st, true);
+    if (rc != ODSGD_OK) return rc;
     cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);
     const bool split = host_local_out && copy_stream && cs != st;
     if (split && (!c->ev_kernel_done || !c->ev_copy_done)) {
@@ -584,7 +780,12 @@ int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, floa
         if (e == cudaSuccess && !c->ev_copy_done) e = cudaEventCreateWithFlags(&c->ev_copy_done, cudaEventDisableTiming);
         if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("event creation: ") + cudaGetErrorString(e));
     }
-    rc = server_call(c, dev_staging, true, worker_id, stream);
+    const size_t bytes = c->n * sizeof(float);
+    for (int m = 0; m < c->n_workers; ++m) {
+        const cudaError_t e = cudaMemcpyAsync(dev_staging[m], host_grads[m], bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("host-to-device copy: ") + cudaGetErrorString(e));
+    }
+    rc = run_server(c, p, st, false);
     if (rc != ODSGD_OK) return rc;
     if (host_local_out) {
         cudaError_t e = cudaSuccess;
@@ -597,6 +798,7 @@ int odsgd_fused_update_host(odsgd_ctx* ctx, const float* const* host_grads, floa
         if (e == cudaSuccess && split) {
             e = cudaEventRecord(c->ev_copy_done, cs);
             c->copy_pending = e == cudaSuccess;
+            c->copy_waited = false;
         }
         if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("device-to-host copy: ") + cudaGetErrorString(e));
     }
@@ -608,10 +810,11 @@ int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stre
     odsgd_ctx* c = ctx;
     if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
     if (!grad) return fail(c, ODSGD_ERR_ARG, "grad is NULL");
-    const size_t bytes = c->n * sizeof(float);
-    const Named g{grad, "grad", -1};
-    for (const Named& s : state_buffers(c))
-        if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, "grad overlaps " + label(s));
+    if (!c->v) return fail(c, ODSGD_ERR_STATE, "a worker-only context (ODSGD_FLAG_WORKER_ONLY) has no server state");
+    StateList st;
+    state_buffers(c, &st);
+    const int rc_o = check_outside(c, st, Named{grad, "grad", -1});
+    if (rc_o != ODSGD_OK) return rc_o;
     AsgdArgs a;
     a.g = grad;
     a.w = c->w[c->cur];
@@ -620,7 +823,11 @@ int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stre
     a.lr = c->lr;
     a.momentum = c->momentum;
     a.wd = c->wd;
-    const int lanes = lanes_for(c, {g, {a.w, "w", -1}, {a.v, "v", -1}});
+    BufList<3> ptrs;
+    ptrs.add(grad, "grad", -1);
+    ptrs.add(a.w, "w", -1);
+    ptrs.add(a.v, "v", -1);
+    const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
     const int rc_dev = on_own_device(c);
     if (rc_dev != ODSGD_OK) return rc_dev;
@@ -662,18 +869,25 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
     if (rule != ODSGD_LOCAL_SGD && rule != ODSGD_LOCAL_DC_C && rule != ODSGD_LOCAL_DC_A && rule != ODSGD_LOCAL_MOMENTUM)
         return fail(c, ODSGD_ERR_ARG, "unknown local rule");
     if (needs_state(rule) && mean_square) {
-        odsgd_ctx probe = *c;
-        for (int w = 0; w < c->n_workers; ++w) probe.mean_square[w] = mean_square[w];
-        const std::vector<Named> st = state_buffers(&probe);
         const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
         for (int w = 0; w < c->n_workers; ++w)
             if (mean_square[w] && !aligned(mean_square[w], need)) return fail(c, ODSGD_ERR_ALIGN, "mean_square arena misaligned");
+        float* keep[ODSGD_MAX_WORKERS];
+        for (int w = 0; w < c->n_workers; ++w) {
+            keep[w] = c->mean_square[w];
+            c->mean_square[w] = mean_square[w];
+        }
+        StateList st;
+        state_buffers(c, &st);
         const int rc = check_distinct(c, st, c->n * sizeof(float));
-        if (rc != ODSGD_OK) return rc;
-        for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = mean_square[w];
+        if (rc != ODSGD_OK) {
+            for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = keep[w];
+            return rc;
+        }
     } else {
         for (int w = 0; w < c->n_workers; ++w) c->mean_square[w] = nullptr;
     }
+    c->state_epoch += 1;  // bound gradient tables were checked against the old set of arenas
     c->local_rule = rule;
     c->dc_lambda = lambda;
     c->dc_m = m;
@@ -684,6 +898,9 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
 int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const float* wd_mult, void* stream) {
     if (!ctx) return ODSGD_ERR_ARG;
     odsgd_ctx* c = ctx;
+    // the table is allocated, filled and freed on the context's own device
+    const int rc_dev = on_own_device(c);
+    if (rc_dev != ODSGD_OK) return rc_dev;
     if (!lr_mult && !wd_mult) {
         if (c->table_dev) cudaFree(c->table_dev);
         c->table_dev = nullptr;
@@ -725,16 +942,19 @@ int odsgd_set_server_mean_square(odsgd_ctx* ctx, float* mean_square) {
     if (mean_square) {
         const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
         if (!aligned(mean_square, need)) return fail(c, ODSGD_ERR_ALIGN, "server mean-square arena misaligned");
-        const size_t bytes = c->n * sizeof(float);
         float* keep = c->server_ms;
         c->server_ms = nullptr;
-        for (const Named& s : state_buffers(c))
-            if (overlap(mean_square, s.p, bytes)) {
+        StateList st;
+        state_buffers(c, &st);
+        const size_t bytes = c->n * sizeof(float);
+        for (int i = 0; i < st.n; ++i)
+            if (overlap(mean_square, st.b[i].p, bytes)) {
                 c->server_ms = keep;
-                return fail(c, ODSGD_ERR_OVERLAP, "server mean-square arena overlaps " + label(s));
+                return fail(c, ODSGD_ERR_OVERLAP, "server mean-square arena overlaps " + label(st.b[i]));
             }
     }
     c->server_ms = mean_square;
+    c->state_epoch += 1;
     return ODSGD_OK;
 }
 
@@ -748,10 +968,10 @@ int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* st
     if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no backup (local) buffer for worker " + std::to_string(worker_id));
     const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
     if (need_ms && !c->server_ms) return fail(c, ODSGD_ERR_STATE, "ODSGD_LOCAL_DC_A at the server needs odsgd_set_server_mean_square");
-    const size_t bytes = c->n * sizeof(float);
-    const Named g{grad, "grad", -1};
-    for (const Named& s : state_buffers(c))
-        if (overlap(g.p, s.p, bytes)) return fail(c, ODSGD_ERR_OVERLAP, "grad overlaps " + label(s));
+    StateList st;
+    state_buffers(c, &st);
+    const int rc_o = check_outside(c, st, Named{grad, "grad", -1});
+    if (rc_o != ODSGD_OK) return rc_o;
     LocalArgs a;
     a.w_bak = c->w[c->cur];
     a.w_out = c->w[c->cur];
@@ -761,8 +981,11 @@ int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* st
     a.n = c->n;
     a.lp = local_params(c);
     a.lp.local_lr = c->lr;  // the server applies its own learning rate
-    std::vector<Named> ptrs = {g, {a.w_out, "w", -1}, {a.x, "local", worker_id}};
-    if (need_ms) ptrs.push_back({a.ms, "server_mean_square", -1});
+    BufList<4> ptrs;
+    ptrs.add(grad, "grad", -1);
+    ptrs.add(a.w_out, "w", -1);
+    ptrs.add(a.x, "local", worker_id);
+    if (need_ms) ptrs.add(a.ms, "server_mean_square", -1);
     const int lanes = lanes_for(c, ptrs);
     if (lanes == 0) return ODSGD_ERR_ALIGN;
     const int rc_copy = before_launch(c, static_cast<cudaStream_t>(stream));
@@ -784,17 +1007,16 @@ int odsgd_set_warmup(odsgd_ctx* ctx, uint64_t wp) {
 
 int odsgd_step(odsgd_ctx* ctx, const float* const* worker_grads, void* stream) {
     if (!ctx) return ODSGD_ERR_ARG;
-    odsgd_ctx* c = ctx;
-    int rc;
-    if (c->iter < c->wp) {
-        rc = server_call(c, worker_grads, false, -2, stream);  // warm-up stage: SSGD
-    } else {
-        // from the last warm-up iteration on: server step + local update of every worker; at
-        // iteration wp itself the gradients were taken on the global weights (no delay yet)
-        rc = server_call(c, worker_grads, true, -1, stream, c->iter == c->wp);
-    }
-    if (rc == ODSGD_OK) c->iter += 1;
-    return rc;
+    return scheduled_step(ctx, [&](bool keep_backup, int local_id, bool first) {
+        return server_call(ctx, worker_grads, keep_backup, local_id, stream, first);
+    });
+}
+
+int odsgd_step_bound(odsgd_ctx* ctx, int slot, void* stream) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    return scheduled_step(ctx, [&](bool keep_backup, int local_id, bool first) {
+        return bound_call(ctx, slot, keep_backup, local_id, stream, first);
+    });
 }
 
 int odsgd_get_train_weights(odsgd_ctx* ctx, int worker_id, float** weights) {
@@ -839,6 +1061,19 @@ float odsgd_lr_poly_decay(float base_lr, float end_lr, float power, uint64_t tot
     if (total_steps == 0 || step >= total_steps) return end_lr;
     const double f = 1.0 - (double)step / (double)total_steps;
     return (float)((double)end_lr + ((double)base_lr - (double)end_lr) * pow(f, (double)power));
+}
+
+int odsgd_shard_range(size_t n_params, int n_ranks, int rank, size_t* begin, size_t* end) {
+    if (!begin || !end || n_ranks < 1 || rank < 0 || rank >= n_ranks) return ODSGD_ERR_ARG;
+    // equal slices of ceil(n / R) elements rounded up to 4 (16 bytes); the last ones ragged or empty
+    const size_t r = (size_t)n_ranks;
+    size_t len = (n_params + r - 1) / r;
+    len = (len + 3) / 4 * 4;
+    const size_t b = len * (size_t)rank;
+    const size_t e = b + len;
+    *begin = b < n_params ? b : n_params;
+    *end = e < n_params ? e : n_params;
+    return ODSGD_OK;
 }
 
 int odsgd_get_weights(odsgd_ctx* ctx, float** current, float** delayed) {
@@ -895,8 +1130,12 @@ namespace {
 constexpr int kMaxDevices = 64;
 unsigned char* g_static_table_addr[kMaxDevices] = {};  // per device: address of g_static_table there
 unsigned char g_static_stage[ODSGD_STATIC_TABLE_BYTES];  // host copy the upload reads from (no allocation)
+// One lock for the address cache and the host staging array: both are shared by every
+// context, device and thread of the process.
+std::mutex g_static_mutex;
 
 // Device address of g_static_table on the current device; looked up on first use.
+// Call with g_static_mutex held.
 int static_table_address(odsgd_ctx* c, unsigned char** out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
@@ -933,54 +1172,34 @@ int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_gr
         return fail(c, ODSGD_ERR_UNSUPPORTED, std::to_string(nt) + " tensors exceed the static table's limit of " +
                                                   std::to_string(ODSGD_STATIC_MAX_TENSORS) +
                                                   " (use odsgd_set_tensor_multipliers + odsgd_fused_update)");
-    bool vec_ok = true;
-    for (size_t o : c->offsets)
-        if (o % 4 != 0) vec_ok = false;
-    if (!vec_ok && !(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED))
+    if (!c->offsets_vec_ok && !(c->flags & ODSGD_FLAG_ALLOW_UNALIGNED))
         return fail(c, ODSGD_ERR_ALIGN, "a tensor offset is not a multiple of 4 elements (set ODSGD_FLAG_ALLOW_UNALIGNED for the scalar path)");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Under stream capture the table upload would become a graph node that re-reads the shared
+    // host staging array at every replay, i.e. whatever table the last eager call of any context
+    // left there: refuse instead.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, ODSGD_ERR_CUDA, "cudaStreamIsCapturing failed");
+    }
+    if (cap != cudaStreamCaptureStatusNone)
+        return fail(c, ODSGD_ERR_STATE, "odsgd_fused_update_mult_static cannot be recorded into a stream capture");
 
-    std::vector<Named> ptrs;
-    int rc = check_grads(c, worker_grads, &ptrs);
+    int rc = check_grads(c, worker_grads);
     if (rc != ODSGD_OK) return rc;
+
+    // From here to the return of the upload the shared host staging array is in use: one call
+    // at a time in the whole process, whatever the device.
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     unsigned char* table = nullptr;
     rc = static_table_address(c, &table);
     if (rc != ODSGD_OK) return rc;
-
-    ServerArgs a;
-    memset(&a, 0, sizeof a);
-    for (int m = 0; m < c->n_workers; ++m) a.g[m] = worker_grads[m];
-    a.v = c->v;
-    a.n = c->n;
-    a.n_workers = c->n_workers;
-    a.inv_n = 1.0f / (float)c->n_workers;
-    a.lr = c->lr;
-    a.momentum = c->momentum;
-    a.wd = c->wd;
-    a.lp = local_params(c);
-    a.w_in = c->w[c->cur];
-    const float* delayed_after = nullptr;
-    int next_cur = c->cur;
-    if (c->pingpong) {
-        a.w_out = c->w[c->cur ^ 1];
-        delayed_after = c->w[c->cur];
-        next_cur = c->cur ^ 1;
-    } else {
-        a.w_out = c->w[c->cur];
-        if (c->w_delayed) {
-            a.w_prev = c->w_delayed;
-            delayed_after = c->w_delayed;
-        }
-    }
-    a.x[0] = c->local[worker_id];
-    a.local_worker = worker_id;
-    ptrs.push_back({a.w_in, "w", -1});
-    ptrs.push_back({a.w_out, "w", -1});
-    ptrs.push_back({a.v, "v", -1});
-    ptrs.push_back({a.x[0], "local", worker_id});
-    if (a.w_prev) ptrs.push_back({a.w_prev, "w_delayed", -1});
-    int lanes = lanes_for(c, ptrs);
-    if (lanes == 0) return ODSGD_ERR_ALIGN;
-    if (!vec_ok) lanes = 1;
+    ServerPlan p;
+    rc = plan_server(c, worker_grads, true, worker_id, false, table, &p);
+    if (rc != ODSGD_OK) return rc;
+    rc = run_server(c, p, st, true);
+    if (rc != ODSGD_OK) return rc;
 
     // table layout: offsets u64 x (T+1) | lr_mult f32 x T | wd_mult f32 x T; every entry the
     // kernel will read is rewritten here, so nothing depends on what an earlier call left
@@ -993,30 +1212,11 @@ int odsgd_fused_update_mult_static(odsgd_ctx* ctx, const float* const* worker_gr
         lm[t] = lr_mult ? lr_mult[t] : 1.0f;
         wm[t] = wd_mult ? wd_mult[t] : 1.0f;
     }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the source is pageable host memory: when this returns, the runtime has taken its own copy
+    // of the bytes, so the staging array may be refilled by the next caller
     const cudaError_t e = cudaMemcpyAsync(table, g_static_stage, bytes, cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return fail(c, ODSGD_ERR_CUDA, std::string("static table upload: ") + cudaGetErrorString(e));
-    a.t_off = reinterpret_cast<const unsigned long long*>(table);
-    a.t_lr_mult = reinterpret_cast<const float*>(table + (nt + 1) * sizeof(unsigned long long));
-    a.t_wd_mult = a.t_lr_mult + nt;
-    a.n_tensors = (unsigned int)nt;
-
-    rc = before_launch(c, st);
-    if (rc != ODSGD_OK) return rc;
-    const bool det = (c->flags & ODSGD_FLAG_ALLOW_FMA) == 0;
-    if (det)
-        rc = lanes == 4 ? launch_server_m<true, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)
-                        : launch_server_m<true, 1, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st);
-    else
-        rc = lanes == 4 ? launch_server_m<false, 4, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st)
-                        : launch_server_m<false, 1, kLocalOne, ODSGD_LOCAL_SGD, true>(c, a, st);
-    if (rc != ODSGD_OK) return rc;
-    c->cur = next_cur;
-    c->step += 1;
-    c->delayed = delayed_after;
-    c->grads_bound = true;
-    for (int m = 0; m < c->n_workers; ++m) c->bound[m] = worker_grads[m];
-    return ODSGD_OK;
+    return run_server(c, p, st, false);
 }
 
 const char* odsgd_last_error(odsgd_ctx* ctx) {

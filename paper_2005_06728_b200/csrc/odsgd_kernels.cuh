@@ -107,6 +107,14 @@ constexpr int kServerCtasPerSm = 64;
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
 
+// Vectors per thread per tile of the server kernel: UB as instantiated, except when the pass
+// also carries every worker's local update (fewer when that update is delay-compensated and
+// touches three arenas per worker: registers are the scarce resource there).  The kernel and
+// the host-side grid sizing both take the tile from here.
+__host__ __device__ constexpr int server_vectors_per_thread(int local_mode, int rule, int ub) {
+    return local_mode != kLocalAll ? ub : (rule != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
+}
+
 struct LocalParams {
     float local_lr;
     float lambda;       // Eq. 4 / Eq. 5 compensation coefficient
@@ -417,9 +425,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
     TensorCursor cur;
-    // vectors per thread: fewer when the pass also carries every worker's delay-compensated
-    // local update (three arenas per worker), where registers are the scarce resource
-    constexpr int UU = LOCAL != kLocalAll ? UB : (RULE != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
+    constexpr int UU = server_vectors_per_thread(LOCAL, RULE, UB);
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * UU;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;

@@ -14,8 +14,8 @@ DEV = "cuda:0"
 POISON = float.fromhex("0x1.fffffcp+100")  # a value no update produces by accident
 GUARD = 64  # floats of guard band on each side of every arena
 
-# Tolerance of the non-deterministic build, derived from its arithmetic.  The default build
-# differs from the one-rounding-per-operator evaluation only where the compiler contracts a
+# Tolerance of the opt-in ODSGD_FLAG_ALLOW_FMA flavour, derived from its arithmetic.  It
+# differs from the default one-rounding-per-operator evaluation only where the compiler contracts a
 # multiply with the following add or subtract; each contraction removes one rounding of
 # relative size 2**-24 of the product it swallows.  The server rule has three candidates
 # (wd*w into d, lr*d or momentum*v into v', nothing into w' = w + v' but v' carries over), the

@@ -9,7 +9,8 @@ Each ``pin_*`` function takes an *implementation* (an object with the methods of
 * an exact rational re-evaluation with explicit fp32 rounding.
 
 The same pins run on the CPU oracle (tests/test_oracle_pins.py), on deliberately
-wrong variants (which must fail), and on the CUDA library (tests/test_gpu_pins.py).
+wrong variants (which must fail), and on the CUDA library (tests/test_gpu_parity.py,
+tests/test_gpu_ext.py).
 """
 from __future__ import annotations
 

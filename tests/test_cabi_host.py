@@ -127,6 +127,55 @@ def test_null_context_is_an_argument_error(lib):
     assert lib.odsgd_get_step(null, None) == binding.ERR_ARG
     assert lib.odsgd_create(None, None) == binding.ERR_ARG
     assert lib.odsgd_last_error(null) is not None
+    assert lib.odsgd_bind_grads(null, None, None) == binding.ERR_ARG
+    assert lib.odsgd_unbind_grads(null, 0) == binding.ERR_ARG
+    assert lib.odsgd_global_update_bound(null, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_fused_update_bound(null, 0, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_ssgd_step_bound(null, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_step_bound(null, 0, None) == binding.ERR_ARG
+    assert lib.odsgd_worker_local_update(null, 0, None, None, 0, None) == binding.ERR_ARG
+
+
+def test_worker_only_flag_lifts_the_momentum_requirement(lib):
+    rc, _, msg = _create(lib, _desc(v=None))
+    assert rc == binding.ERR_ARG and "NULL" in msg
+    rc, _, msg = _create(lib, _desc(v=None, flags=binding.FLAG_WORKER_ONLY))
+    # a valid worker-role description gets as far as the device query (no GPU here) or succeeds
+    assert rc in (binding.OK, binding.ERR_CUDA), msg
+    rc, _, msg = _create(lib, _desc(w_a=None, v=None, flags=binding.FLAG_WORKER_ONLY))
+    assert rc == binding.ERR_ARG
+
+
+def _covers(n, ranks):
+    prev_end, lens = 0, []
+    for r in range(ranks):
+        b, e = binding.shard_range(n, ranks, r)
+        assert b == prev_end, "slices are ascending and leave no gap"
+        assert b <= e <= n
+        assert b % 4 == 0 or b == n, "every non-empty slice starts on a 16-byte boundary"
+        prev_end = e
+        lens.append(e - b)
+    assert prev_end == n, "the slices cover the arena exactly"
+    return lens
+
+
+def test_shard_ranges_partition_the_arena():
+    """odsgd_shard_range: equal 16-byte-aligned slices, ragged (or empty) at the end."""
+    for n in (1, 3, 4, 5, 7, 8, 33, 1000, 1023, 1024, 1025, 431_080, 853_018, 60_965_224, 25_557_032, 138_357_544,
+              (1 << 32) + 5):
+        for ranks in (1, 2, 3, 4, 7, 8, 16, 64):
+            lens = _covers(n, ranks)
+            nominal = -(-(-(-n // ranks)) // 4) * 4  # ceil(ceil(n / R) / 4) * 4
+            full = [x for x in lens if x == nominal]
+            ragged = [x for x in lens if 0 < x < nominal]
+            assert len(ragged) <= 1 and len(full) + len(ragged) + lens.count(0) == ranks
+            assert lens == sorted(lens, reverse=True), "full slices first, then the ragged one, then empty ones"
+    assert binding.shard_range(10, 4, 0) == (0, 4) and binding.shard_range(10, 4, 2) == (8, 10)
+    assert binding.shard_range(10, 4, 3) == (10, 10), "more ranks than 4-element groups: trailing slices are empty"
+    assert binding.shard_range(138_357_544, 8, 7) == (7 * 17_294_696, 138_357_544)
+    for bad in ((10, 0, 0), (10, 2, 2), (10, 2, -1)):
+        with pytest.raises(binding.OdsgdError):
+            binding.shard_range(*bad)
 
 
 def test_missing_library_fails_loudly(tmp_path):

@@ -1,8 +1,9 @@
 """CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200).
 
-Bars: bit-exact in the deterministic build flavour (ODSGD_FLAG_DETERMINISTIC); within
-gpu_util.REL_TOL of the oracle, relative to the magnitude of the terms each element is built
-from, in the default flavour (where multiply-add pairs may be fused).
+Bars: bit-exact in the default flavour (flags = 0, or ODSGD_FLAG_DETERMINISTIC spelled out:
+one rounding per operator); within gpu_util.REL_TOL of the oracle, relative to the magnitude of
+the terms each element is built from, in the opt-in ODSGD_FLAG_ALLOW_FMA flavour (where
+multiply-add pairs may be fused).
 """
 import numpy as np
 import pytest
@@ -36,7 +37,7 @@ def test_pins_on_gpu_fused_kernel(cuda_device, pin):
 @pytest.mark.parametrize("pin", [pins.pin_worked_example, pins.pin_dc_worked_example,
                                  pins.pin_ssgd_quadratic_closed_form, pins.pin_odsgd_quadratic_matrix_form,
                                  pins.pin_special_values], ids=lambda f: f.__name__)
-def test_pins_on_gpu_default_build(cuda_device, pin):
+def test_pins_on_gpu_fma_flavour(cuda_device, pin):
     # dyadic examples and closed forms hold with or without fused multiply-add
     pin(GpuImpl(deterministic=False))
 
@@ -148,7 +149,7 @@ def test_fused_all_locals_bit_exact(cuda_device, nw):
 
 
 @pytest.mark.parametrize("n", [1, 5, 1025, 70_001])
-def test_default_build_within_tolerance(cuda_device, n):
+def test_fma_flavour_within_tolerance(cuda_device, n):
     for nw in (1, 4, 9):
         w, v, grads = _case(n, nw, seed=n + 7 * nw)
         wo, vo, wp, xs = _oracle_fused(w, v, grads, HP)
@@ -408,14 +409,14 @@ def test_lenet5_full_run_bit_exact(cuda_device):
     _trajectory(wl, True, wl.iterations)
 
 
-def test_lenet5_full_run_default_build(cuda_device):
+def test_lenet5_full_run_fma_flavour(cuda_device):
     wl = W.workload("lenet5")
     worst, (ctx, w_ref, v_ref) = _trajectory(wl, False, wl.iterations)
     assert max(worst.values()) <= 1e-6
     # reported, not gated: error relative to the result itself (floored per tensor), which
     # cancellation between the momentum and gradient terms can inflate
     rel, over = plain_relative_error(ctx.weights().cpu().numpy(), w_ref, wl.offsets)
-    print(f"lenet5 default build: plain relative error max {rel:.3e}, {over} elements above 1e-6")
+    print(f"lenet5 FMA flavour: plain relative error max {rel:.3e}, {over} elements above 1e-6")
     assert np.isfinite(rel)
 
 
@@ -424,13 +425,13 @@ def test_resnet56_full_run_bit_exact(cuda_device):
     _trajectory(wl, True, wl.iterations, check_every=10)
 
 
-def test_resnet56_default_build(cuda_device):
+def test_resnet56_fma_flavour(cuda_device):
     wl = W.workload("resnet56")
     worst, _ = _trajectory(wl, False, 20, check_every=5)
     assert max(worst.values()) <= 1e-6
 
 
-def test_free_running_default_build_stays_close(cuda_device):
+def test_free_running_fma_flavour_stays_close(cuda_device):
     """Both sides free-running for the whole run: rounding differences may accumulate, but slowly."""
     wl = W.workload("lenet5")
     ctx, w, v, local = _ctx_for(wl, False, True)
