@@ -11,9 +11,14 @@ step, with every buffer resident in HBM; `e2e` is the same figure when the M gra
 in pinned host memory and the worker's new weights are copied back, all inside the timed
 region, through the host-buffer entry point of the C ABI.  One JSON line goes to stdout.
 
-With --gpus N > 1 (under torchrun) every rank updates its own full parameter set on its own
-GPU: the ranks share no data, so nothing but a barrier and the final max/sum of two scalars
-crosses between them.
+Besides the headline workload (VGG-16-shaped, M = 32) the default run times, and reports under
+`configs`, the other parameter sets: every rule on the AlexNet- and ResNet-50-shaped sets, the
+worker-count sweep on the VGG-16-shaped set, and the two small cache-resident sets (eager
+launches and CUDA-graph replay; effective figures, not HBM ones).
+
+With --gpus N > 1 every rank updates its own full parameter set on its own GPU: the ranks share
+no data, so nothing but a barrier and the final max/sum of two scalars crosses between them.
+Started without torchrun, `--gpus N` launches its N ranks itself.
 """
 from __future__ import annotations
 
@@ -21,6 +26,7 @@ import argparse
 import json
 import os
 import statistics
+import subprocess
 import sys
 import time
 
@@ -30,6 +36,8 @@ sys.path.insert(0, ROOT)
 METRIC = "OD-SGD update throughput: HBM GB/s & % of B200 peak; params/sec at N workers"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126e6
+ORACLE_CHUNK = 1 << 22  # elements per chunk when the oracle walks a whole arena
 
 
 def hbm_peak():
@@ -64,7 +72,7 @@ def workload_label(wl, n_workers):
     return f"{wl.name}-shaped parameter set, M={n_workers} workers, fused global+local update"
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=400)
@@ -85,11 +93,32 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra-kernels", action="store_true")
-    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="elements in the oracle's sample")
-    return ap.parse_args()
+    ap.add_argument("--no-configs", action="store_true", help="skip the other parameter sets (only the headline workload)")
+    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="elements in the reference arm's sample")
+    return ap.parse_args(argv)
 
 
 # ----------------------------------------------------------------------------- CPU oracle arm
+class _OneCore:
+    """Pins the process to one core while the single-threaded oracle is timed."""
+
+    def __enter__(self):
+        self.old = None
+        try:
+            self.old = os.sched_getaffinity(0)
+            os.sched_setaffinity(0, {sorted(self.old)[-1]})
+        except (AttributeError, OSError):
+            self.old = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.old:
+            try:
+                os.sched_setaffinity(0, self.old)
+            except OSError:
+                pass
+
+
 def oracle_sample(wl, n_workers, sample_elems):
     """Inputs for the oracle: the workload's hyper-parameters and value distributions on an
     arena cut down to `sample_elems` elements."""
@@ -109,7 +138,7 @@ def oracle_sample(wl, n_workers, sample_elems):
 
 
 def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
-    """Times the oracle as it stands (single thread) on the sample; returns (GB/s, info)."""
+    """Times the oracle as it stands (single thread) on a sample made on the host."""
     import numpy as np
 
     import oracle
@@ -117,30 +146,20 @@ def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
 
     cut, w, v, grads = oracle_sample(wl, n_workers, sample_elems)
     s = w.size
-    old_affinity = None
-    try:  # one core, as the oracle is single-threaded; keeps the figure free of migrations
-        old_affinity = os.sched_getaffinity(0)
-        os.sched_setaffinity(0, {sorted(old_affinity)[-1]})
-    except (AttributeError, OSError):
-        old_affinity = None
     wp = np.empty_like(w)
     x = np.empty_like(w)
     times = []
-    t_start = time.perf_counter()
-    for it in range(warmup + steps):
-        t0 = time.perf_counter()
-        oracle.global_update(grads, w, v, lr=wl.lr, momentum=wl.momentum, wd=wl.wd, w_prev=wp)
-        oracle.local_update(wp, grads[0], local_lr=wl.local_lr, out=x)
-        dt = time.perf_counter() - t0
-        if it >= warmup:
-            times.append(dt)
-        if it >= warmup + 2 and time.perf_counter() - t_start > budget_s:
-            break
-    if old_affinity:
-        try:
-            os.sched_setaffinity(0, old_affinity)
-        except OSError:
-            pass
+    with _OneCore():
+        t_start = time.perf_counter()
+        for it in range(warmup + steps):
+            t0 = time.perf_counter()
+            oracle.global_update(grads, w, v, lr=wl.lr, momentum=wl.momentum, wd=wl.wd, w_prev=wp)
+            oracle.local_update(wp, grads[0], local_lr=wl.local_lr, out=x)
+            dt = time.perf_counter() - t0
+            if it >= warmup:
+                times.append(dt)
+            if it >= warmup + 2 and time.perf_counter() - t_start > budget_s:
+                break
     sec = statistics.median(times)
     nbytes = algorithmic_bytes("fused", s, n_workers)
     info = {"value": nbytes / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
@@ -148,6 +167,52 @@ def time_oracle(wl, n_workers, sample_elems, steps, warmup, budget_s=25.0):
                       f"{len(times)} calls of global+local update, single thread",
             "ms_per_call": sec * 1e3, "params_per_s": s / sec, "host": host_info()}
     return info, len(times), sec
+
+
+def time_oracle_full(wl, n_workers, w_dev, grads_dev, passes=3):
+    """Times the oracle as it stands (single thread) on the WHOLE arena of the workload: the
+    benchmark's own device-resident inputs are brought to the host chunk by chunk (outside the
+    timed sections; the rules are element-wise, so the oracle's loops are unchanged) and a pass
+    is the sum of the oracle's time over all chunks.  Median of `passes` passes after a warm-up
+    on the first chunk."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes, host_info
+
+    n = wl.arena_len
+    ch = min(ORACLE_CHUNK, n)
+    stage = torch.empty((n_workers, ch), dtype=torch.float32).pin_memory()
+    w = w_dev.cpu().numpy().copy()
+    v = np.zeros(n, np.float32)
+    wp = np.empty(ch, np.float32)
+    x = np.empty(ch, np.float32)
+    hp = dict(lr=wl.lr, momentum=wl.momentum, wd=wl.wd)
+    totals = []
+    with _OneCore():
+        for p in range(passes + 1):
+            total = 0.0
+            for a in range(0, n, ch):
+                b = min(a + ch, n)
+                for m in range(n_workers):
+                    stage[m, :b - a].copy_(grads_dev[m][a:b], non_blocking=True)
+                torch.cuda.synchronize()
+                gh = [stage[m, :b - a].numpy() for m in range(n_workers)]
+                t0 = time.perf_counter()
+                oracle.global_update(gh, w[a:b], v[a:b], w_prev=wp[:b - a], **hp)
+                oracle.local_update(wp[:b - a], gh[0], local_lr=wl.local_lr, out=x[:b - a])
+                total += time.perf_counter() - t0
+                if p == 0:
+                    break  # warm-up: one chunk touches every buffer the later passes use
+            if p > 0:
+                totals.append(total)
+    sec = statistics.median(totals)
+    nbytes = algorithmic_bytes("fused", wl.n_params, n_workers)
+    return {"value": nbytes / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"the whole {wl.name} arena ({n} elements, all {n_workers} workers), walked in chunks of "
+                      f"{ch} elements; median of {passes} passes of global+local update, single thread",
+            "ms_per_call": sec * 1e3, "params_per_s": wl.n_params / sec, "host": host_info()}
 
 
 def run_reference(args):
@@ -175,6 +240,161 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+def _timed(fn, reps, stream, warm=3):
+    """ms per call: CUDA events on the launching stream around `reps` back-to-back calls."""
+    import torch
+
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(reps):
+        fn()
+    b.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def _rate(nbytes, ms, peak, hbm_bound=True):
+    gbps = nbytes / ms / 1e6
+    return {"ms": ms, "GBps": gbps, "frac": gbps / peak if hbm_bound else None,
+            "frac_of_nominal_8000": gbps / NOMINAL_HBM_GBS if hbm_bound else None}
+
+
+class _Set:
+    """One parameter set resident on the device, with a context over it."""
+
+    def __init__(self, wl, M, dev, flags=0, n_locals=1):
+        import torch
+
+        from paper_2005_06728_b200 import binding
+        from paper_2005_06728_b200 import workloads as W
+
+        self.wl, self.M, self.dev = wl, M, dev
+        self.w_a = W.make_weights(wl, dev)
+        self.w_b = torch.zeros_like(self.w_a)
+        self.v = W.make_momentum(wl, dev)
+        self.local = [self.w_a.clone() for _ in range(n_locals)] + [None] * (M - n_locals)
+        self.sg, self.pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
+        self.grads = [W.make_grad(wl, m, 0, dev, _sigma=self.sg, _pads=self.pads) for m in range(M)]
+        self.flags = flags
+        self.ctx = binding.Odsgd(self.w_a, self.v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum,
+                                 wd=wl.wd, w_b=self.w_b, local=self.local, tensor_offsets=wl.offsets, flags=flags)
+
+    def sub_context(self, m):
+        """A context over the first m gradient buffers of the same arenas (worker sweep)."""
+        from paper_2005_06728_b200 import binding
+
+        wl = self.wl
+        return binding.Odsgd(self.w_a, self.v, n_workers=m, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum,
+                             wd=wl.wd, w_b=self.w_b, local=[self.local[0]] + [None] * (m - 1),
+                             tensor_offsets=wl.offsets, flags=self.flags)
+
+
+def _all_rules(s, reps, stream, peak, hbm_bound=True):
+    """ms and GB/s of every rule on one resident set (bound gradient table, back-to-back calls)."""
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes
+
+    ctx, P, M = s.ctx, s.wl.n_params, s.M
+    bound = ctx.bind_grads(s.grads)
+    out = {}
+    calls = (("fused", lambda: ctx.fused_update(bound, 0, stream)),
+             ("global", lambda: ctx.global_update(bound, stream)),
+             ("local", lambda: ctx.local_update(0, stream)),
+             ("ssgd", lambda: ctx.ssgd_step(bound, stream)),
+             ("asgd", lambda: ctx.asgd_step(0, s.grads[0], stream)))
+    for name, fn in calls:
+        if name == "local":
+            ctx.global_update(bound, stream)
+        out[name] = _rate(algorithmic_bytes(name, P, M), _timed(fn, reps, stream), peak, hbm_bound)
+    bound.unbind()
+    return out
+
+
+def _sweep(s, worker_counts, reps, stream, peak):
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes
+
+    rows = []
+    for m in worker_counts:
+        if m < 1 or m > s.M:
+            continue
+        c2 = s.sub_context(m)
+        bound = c2.bind_grads(s.grads[:m])
+        ms = _timed(lambda: c2.fused_update(bound, 0, stream), reps, stream)
+        nb = algorithmic_bytes("fused", s.wl.n_params, m)
+        row = {"workers": m, "bytes_per_step": nb, "params_per_s": s.wl.n_params / (ms * 1e-3),
+               "grad_elems_per_s": m * s.wl.n_params / (ms * 1e-3)}
+        row.update(_rate(nb, ms, peak))
+        rows.append(row)
+        c2.close()
+    return rows
+
+
+def _small_set_entry(name, dev, stream, flags, steps=4000, graph_steps=20):
+    """A cache-resident set: eager launches through the bound-table call, and CUDA-graph replay."""
+    import torch
+
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes
+
+    wl = W.workload(name)
+    s = _Set(wl, wl.n_workers, dev, flags)
+    ctx = s.ctx
+    bound = ctx.bind_grads(s.grads)
+    sh = stream.cuda_stream
+    raw, slot = ctx.fused_update_bound_raw, bound.slot
+    rcs = []
+    eager_ms = _timed(lambda: rcs.append(raw(slot, 0, sh)), steps, stream, warm=20)
+    bad = [rc for rc in rcs if rc != 0]
+    if bad:
+        ctx.check(bad[0])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(graph_steps):
+            ctx.fused_update(bound, 0)
+    graph_ms = _timed(graph.replay, max(1, steps // graph_steps), stream) / graph_steps
+    nb = algorithmic_bytes("fused", wl.n_params, wl.n_workers)
+    entry = {"workload": workload_label(wl, wl.n_workers), "n_params": wl.n_params, "n_tensors": wl.n_tensors,
+             "n_workers": wl.n_workers, "bytes_per_step": nb,
+             "l2": "effective, L2-resident: the working set fits in the 126 MB L2, so these are not HBM figures",
+             "fused": {"eager_us_per_step": eager_ms * 1e3, "eager_effective_GBps": nb / eager_ms / 1e6,
+                       "graph_us_per_step": graph_ms * 1e3, "graph_effective_GBps": nb / graph_ms / 1e6,
+                       "frac": None, "steps": steps,
+                       "launch": "eager: odsgd_fused_update_bound from a Python loop, one launch per step; "
+                                 f"graph: {graph_steps} steps captured once and replayed"},
+             "params_per_s": wl.n_params / (eager_ms * 1e-3)}
+    bound.unbind()
+    rules = _all_rules(s, 200, stream, 1.0, hbm_bound=False)
+    for k, r in rules.items():
+        if k != "fused":
+            entry[k] = {"us": r["ms"] * 1e3, "effective_GBps": r["GBps"], "frac": None}
+    ctx.close()
+    return entry
+
+
+def _large_set_entry(name, dev, stream, flags, peak, reps, cpu_full):
+    import torch
+
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import algorithmic_bytes
+
+    wl = W.workload(name)
+    s = _Set(wl, wl.n_workers, dev, flags)
+    entry = {"workload": workload_label(wl, wl.n_workers), "n_params": wl.n_params, "n_tensors": wl.n_tensors,
+             "n_workers": wl.n_workers, "bytes_per_step": algorithmic_bytes("fused", wl.n_params, wl.n_workers),
+             "l2": "inputs per step exceed the 126 MB L2 many times over: no flush", "reps": reps}
+    entry.update(_all_rules(s, reps, stream, peak))
+    entry["params_per_s"] = wl.n_params / (entry["fused"]["ms"] * 1e-3)
+    entry["grad_elems_per_s"] = wl.n_workers * entry["params_per_s"]
+    if cpu_full:
+        entry["cpu_oracle_full"] = time_oracle_full(wl, wl.n_workers, s.w_a, s.grads)
+    s.ctx.close()
+    del s
+    torch.cuda.empty_cache()
+    return entry
+
+
 def run_cuda(args):
     import torch
 
@@ -206,17 +426,12 @@ def run_cuda(args):
     if need > 0.9 * free:
         raise SystemExit(f"{wl.name} with {M} workers needs {need / 2**30:.1f} GiB; {free / 2**30:.1f} GiB free")
 
-    w_a = W.make_weights(wl, dev)
-    w_b = torch.zeros_like(w_a)
-    v = W.make_momentum(wl, dev)
+    flags = binding.FLAG_ALLOW_FMA if args.allow_fma else 0
     n_locals = M if args.all_locals else 1
     wid = -1 if args.all_locals else 0
-    local = [w_a.clone() for _ in range(n_locals)] + [None] * (M - n_locals)
-    sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
-    grads = [W.make_grad(wl, m, 0, dev, _sigma=sg, _pads=pads) for m in range(M)]
-    flags = binding.FLAG_ALLOW_FMA if args.allow_fma else 0
-    ctx = binding.Odsgd(w_a, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
-                        w_b=w_b, local=local, tensor_offsets=wl.offsets, flags=flags)
+    head = _Set(wl, M, dev, flags, n_locals)
+    ctx, local, grad_list = head.ctx, head.local, head.grads
+    w_a = head.w_a
     if args.block or args.ctas_per_sm:
         ctx.set_launch_config(args.block, args.ctas_per_sm)
     stream = torch.cuda.current_stream()
@@ -231,9 +446,9 @@ def run_cuda(args):
         ctx.set_tensor_multipliers(None, [1.0 if t.kind == "weight" else 0.0 for t in wl.tensors])
 
     step_bytes = algorithmic_bytes("fused", P, M, n_locals) + extra_streams * 4 * P
-    grad_list = grads
-    grads = ctx.grad_table(grad_list)  # pointers marshalled once, as a training loop would
-    l2_note = ("inputs per step exceed the 126 MB L2 many times over: no flush" if step_bytes > 8 * 126e6
+    hbm_bound = step_bytes > 8 * L2_BYTES
+    grads = ctx.bind_grads(grad_list)  # validated once, as a training loop would
+    l2_note = ("inputs per step exceed the 126 MB L2 many times over: no flush" if hbm_bound
                else "working set fits in L2: effective GB/s, not an HBM figure")
 
     for _ in range(max(3, args.warmup)):
@@ -252,31 +467,38 @@ def run_cuda(args):
         torch.cuda.synchronize()
     barrier(dev)
     torch.cuda.synchronize()
-    launches_before = ctx.launch_count
     if graph is None:
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        # an event after every step for steps of half a millisecond or more; for short steps (where
+        # the event itself would cost as much as the step) one every `stride` steps
+        probe_ms = _timed(lambda: ctx.fused_update(grads, wid, stream), 4, stream, warm=0)
+        stride = 1 if probe_ms >= 0.5 else max(1, min(50, args.steps // 8))
+        marks = list(range(0, args.steps, stride)) + [args.steps]
+        ev = {k: torch.cuda.Event(enable_timing=True) for k in marks}
+        launches_before = ctx.launch_count
         with ClockSampler(dev.index or 0) as clocks:
             ev[0].record(stream)
             for k in range(args.steps):
                 ctx.fused_update(grads, wid, stream)
-                ev[k + 1].record(stream)
+                if k + 1 in ev:
+                    ev[k + 1].record(stream)
             torch.cuda.synchronize()
         gpu_launches = ctx.launch_count - launches_before
-        per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+        per_step = [ev[a].elapsed_time(ev[b]) / (b - a) for a, b in zip(marks[:-1], marks[1:])]
+        total_ms = ev[0].elapsed_time(ev[args.steps])
     else:
         replays = args.steps // args.graph
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
+        evl = [torch.cuda.Event(enable_timing=True) for _ in range(replays + 1)]
         with ClockSampler(dev.index or 0) as clocks:
-            ev[0].record(stream)
+            evl[0].record(stream)
             for k in range(replays):
                 graph.replay()
-                ev[k + 1].record(stream)
+                evl[k + 1].record(stream)
             torch.cuda.synchronize()
         gpu_launches = args.steps  # one kernel node per captured step, replayed
-        per_step = [ev[k].elapsed_time(ev[k + 1]) / args.graph for k in range(replays)]
+        per_step = [evl[k].elapsed_time(evl[k + 1]) / args.graph for k in range(replays)]
+        total_ms = evl[0].elapsed_time(evl[-1])
     barrier(dev)
     torch.cuda.synchronize()
-    total_ms = ev[0].elapsed_time(ev[-1])
     agg = aggregate(total_ms, float(step_bytes) * args.steps, dev if world > 1 else None)
     ms_per_step = agg["ms"] / args.steps
     value = agg["units"] / (agg["ms"] * 1e-3) / 1e9
@@ -287,18 +509,6 @@ def run_cuda(args):
     # ---- the other rules on the same arena (context only; not part of `value`)
     extra = {}
     if not args.no_extra_kernels and rank0:
-        def timed(fn, reps):
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for _ in range(reps):
-                fn()
-            b.record(stream)
-            torch.cuda.synchronize()
-            return a.elapsed_time(b) / reps
-
         reps = max(5, min(50, args.steps))
         for name, fn in (("global", lambda: ctx.global_update(grads, stream)),
                          ("local", lambda: ctx.local_update(0, stream)),
@@ -306,39 +516,18 @@ def run_cuda(args):
                          ("asgd", lambda: ctx.asgd_step(0, grad_list[0], stream))):
             if name == "local":
                 ctx.global_update(grads, stream)
-            ms = timed(fn, reps)
-            b = algorithmic_bytes(name, P, M)
-            extra[name] = {"ms": ms, "GBps": b / ms / 1e6, "frac": b / ms / 1e6 / peak}
+            extra[name] = _rate(algorithmic_bytes(name, P, M), _timed(fn, reps, stream), peak, hbm_bound)
 
     # ---- worker-count sweep on the same arena (fused update, first m gradient buffers)
-    sweep = []
-    if args.sweep_workers and rank0:
-        for m in [int(x) for x in args.sweep_workers.split(",") if x]:
-            if m < 1 or m > M:
-                continue
-            loc = [local[0]] + [None] * (m - 1)
-            c2 = binding.Odsgd(w_a, v, n_workers=m, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
-                               w_b=w_b, local=loc, tensor_offsets=wl.offsets, flags=flags)
-            reps = max(20, min(200, args.steps))
-            for _ in range(3):
-                c2.fused_update(grad_list[:m], 0, stream)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            for _ in range(reps):
-                c2.fused_update(grad_list[:m], 0, stream)
-            b.record(stream)
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / reps
-            nb = algorithmic_bytes("fused", P, m)
-            sweep.append({"workers": m, "ms": ms, "GBps": nb / ms / 1e6, "frac": nb / ms / 1e6 / peak,
-                          "params_per_s": P / (ms * 1e-3), "bytes_per_step": nb})
-            c2.close()
+    sweep_counts = [int(x) for x in args.sweep_workers.split(",") if x]
+    if not sweep_counts and not args.no_configs and args.workload == "vgg16" and not args.workers:
+        sweep_counts = [1, 2, 4, 8, 16, 32]
+    sweep = _sweep(head, sweep_counts, max(20, min(200, args.steps)), stream, peak) if sweep_counts and rank0 else []
 
     # ---- end to end: gradients start in pinned host memory, local weights come back
     e2e = None
     if not args.no_e2e:
-        pool = [W.make_grad(wl, m, 1, dev, _sigma=sg, _pads=pads).cpu().pin_memory() for m in range(min(M, 4))]
+        pool = [W.make_grad(wl, m, 1, dev, _sigma=head.sg, _pads=head.pads).cpu().pin_memory() for m in range(min(M, 4))]
         host_grads = [pool[m % len(pool)] for m in range(M)]
         host_out = torch.empty(n, dtype=torch.float32).pin_memory()
         e2e_steps = max(2, min(args.steps, 6))
@@ -360,23 +549,43 @@ def run_cuda(args):
         wall_ms = (time.perf_counter() - t0) * 1e3
         e2e_ms = max(a.elapsed_time(b), wall_ms)
         agg2 = aggregate(e2e_ms, float(step_bytes) * e2e_steps, dev if world > 1 else None)
+        h2d, d2h = M * n * 4, n * 4
         e2e = {"value": agg2["units"] / (agg2["ms"] * 1e-3) / 1e9, "unit": "GB/s",
-               "h2d_bytes_per_step": M * n * 4, "d2h_bytes_per_step": n * 4, "steps": e2e_steps,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "ms_per_step": agg2["ms"] / e2e_steps,
+               "h2d_GBps": h2d * e2e_steps * world / (agg2["ms"] * 1e-3) / 1e9,
+               "what": "ALGORITHMIC bytes of the update, (M + 5) * 4 * P per step, over a time that is set by the "
+                       "host link: M * 4 * P bytes cross it per step (h2d_GBps is that traffic over the same time), "
+                       "so this figure may sit above what the bus itself carries",
                "note": f"{M} host-to-device copies per step from a pool of {len(pool)} distinct pinned buffers; "
                        + ("copy-back of the local weights on a second stream" if copy_stream is not None
                           else "copy-back on the same stream (small arena)")}
+        del pool, host_grads, host_out
 
     if not rank0:
         return 0
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        info, _, _ = time_oracle(wl, M, args.cpu_sample, steps=10, warmup=1)
-        cpu = {k: info[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        info = time_oracle_full(wl, M, w_a, grad_list)
+        cpu = {k: info[k] for k in ("value", "unit", "cores", "kind", "sample", "ms_per_call")}
         cpu["host"] = info["host"]
 
+    # ---- the other parameter sets (reported under `configs`; not part of `value`)
+    configs = []
+    if not args.no_configs and world == 1 and args.workload == "vgg16" and not args.workers:
+        grads.unbind()
+        ctx.close()
+        del head, ctx, local, grad_list, grads, w_a
+        torch.cuda.empty_cache()
+        for name in ("alexnet", "resnet50"):
+            configs.append(_large_set_entry(name, dev, stream, flags, peak, reps=200,
+                                            cpu_full=not args.no_cpu_baseline))
+        for name in ("resnet56", "lenet5"):
+            configs.append(_small_set_entry(name, dev, stream, flags))
+
     ck = clocks.summary()
+    roof_frac = achieved / peak if hbm_bound else None
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -391,9 +600,11 @@ def run_cuda(args):
         "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),
                    "power_w_max": ck.get("power_w_max"), "samples": ck.get("samples"), "source": ck.get("source")},
         "e2e": e2e, "gpu_launches": gpu_launches,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": measured_traffic(step_bytes), "peak_source": f"of {peak_src}", "kernel": "server_kernel (fused, one local)",
-                     "kernel_ms": kernel_ms, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": roof_frac,
+                     "traffic": measured_traffic(step_bytes) if hbm_bound else None, "peak_source": f"of {peak_src}",
+                     "kernel": "server_kernel (fused, one local)", "kernel_ms": kernel_ms,
+                     "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS if hbm_bound else None,
+                     "note": None if hbm_bound else "cache-resident working set: effective GB/s, no HBM fraction"},
         "cpu_baseline": cpu,
         "params_per_s": P * args.steps * world / (agg["ms"] * 1e-3),
         "grad_elems_per_s": M * P * args.steps * world / (agg["ms"] * 1e-3),
@@ -402,12 +613,40 @@ def run_cuda(args):
     }
     if sweep:
         line["worker_sweep"] = sweep
+    if configs:
+        line["configs"] = configs
     print(json.dumps(line), flush=True)
     return 0
 
 
-def main():
-    args = parse_args()
+# ----------------------------------------------------------------------------- launching N ranks
+def self_launch_command(argv, n_gpus, port):
+    """The torchrun command line that runs this script as `n_gpus` ranks on this node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"), *argv]
+
+
+def self_launch(argv, n_gpus):
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    return subprocess.run(self_launch_command(argv, n_gpus, port), cwd=ROOT).returncode
+
+
+def main(argv=None):
+    argv = list(sys.argv[1:] if argv is None else argv)
+    args = parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: become the launcher of the N ranks (each re-enters main() under torchrun)
+        if args.impl == "cuda":
+            import torch
+
+            have = torch.cuda.device_count()
+            if have < args.gpus:
+                raise SystemExit(f"--gpus {args.gpus}: only {have} CUDA device(s) visible")
+        return self_launch(argv, args.gpus)
     if args.impl == "reference":
         return run_reference(args)
     try:

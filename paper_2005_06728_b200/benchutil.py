@@ -42,7 +42,7 @@ class ClockSampler:
     setting.  Use as a context manager around the timed region.
     """
 
-    def __init__(self, cuda_index: int = 0, period_s: float = 0.02):
+    def __init__(self, cuda_index: int = 0, period_s: float = 0.005):
         self.cuda_index = cuda_index
         self.period_s = period_s
         self.samples: List[Dict] = []

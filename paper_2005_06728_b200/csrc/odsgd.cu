@@ -216,6 +216,24 @@ int on_own_device(odsgd_ctx* c) {
     return ODSGD_OK;
 }
 
+// One launch on `st`, marked so that it may be scheduled while the kernel ahead of it in the
+// stream is still draining (the kernels themselves wait for that kernel's completion before
+// they touch memory).
+template <typename Args>
+void launch_kernel(void (*kernel)(const Args), int grid, int block, cudaStream_t st, const Args& a) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3((unsigned)block, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = kProgrammaticLaunch ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, a);  // the error, if any, is picked up by after_launch
+}
+
 int too_wide(odsgd_ctx* c, int block) {
     return fail(c, ODSGD_ERR_UNSUPPORTED, "block_threads = " + std::to_string(block) + " is too large for this kernel");
 }
@@ -229,7 +247,7 @@ int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     if (dry) return ODSGD_OK;
     const int grid = grid_for(c, a.n, NL, block, server_vectors_per_thread(LOCAL, RULE, UB), kServerCtasPerSm);
-    kernel<<<grid, block, 0, st>>>(a);
+    launch_kernel<ServerArgs>(kernel, grid, block, st, a);
     return after_launch(c, "server kernel launch");
 }
 
@@ -283,7 +301,7 @@ int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = local_kernel<DET, NL, RULE, SERVER>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
+    launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, st, a);
     return after_launch(c, "local kernel launch");
 }
 
@@ -312,7 +330,7 @@ int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
     auto kernel = asgd_kernel<DET, NL>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    kernel<<<grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, 0, st>>>(a);
+    launch_kernel<AsgdArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, st, a);
     return after_launch(c, "asgd kernel launch");
 }
 

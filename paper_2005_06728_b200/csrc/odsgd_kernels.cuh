@@ -17,6 +17,13 @@
 //   * a grid of SMs x 64 CTAs at most strides over the tiles, so one launch
 //     covers the whole arena whatever the number of tensors in it, and the
 //     hardware scheduler evens out the tail.
+//   * every kernel opens with the two programmatic-dependent-launch instructions: it lets the
+//     next kernel of the stream be scheduled at once (griddepcontrol.launch_dependents) and
+//     itself waits, before its first memory access, until the kernels ahead of it have
+//     completed and their writes are visible (griddepcontrol.wait).  Launched with the
+//     matching attribute, back-to-back update kernels no longer pay the full launch latency
+//     between them, which is most of an iteration on the small, cache-resident parameter sets;
+//     launched without it, both instructions do nothing.
 // Tensor cores have no role here: there is no contraction.
 #pragma once
 
@@ -164,6 +171,18 @@ struct AsgdArgs {
     unsigned long long n;
     float lr, momentum, wd;
 };
+
+// ------------------------------------------------------------------ dependent launch
+// 1: launch with programmatic stream serialization (0 keeps the instructions, drops the attribute).
+#ifndef ODSGD_PDL
+#define ODSGD_PDL 1
+#endif
+constexpr bool kProgrammaticLaunch = ODSGD_PDL != 0;
+
+__device__ __forceinline__ void dependent_launch_prologue() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 
 // ------------------------------------------------------------------ vectors
 template <int NL>
@@ -424,6 +443,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 // warps, more vectors per thread) measured 7-20 % faster.
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
+    dependent_launch_prologue();
     TensorCursor cur;
     constexpr int UU = server_vectors_per_thread(LOCAL, RULE, UB);
     const unsigned long long nvec = a.n / NL;
@@ -485,6 +505,7 @@ __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned
 
 template <bool DET, int NL, int RULE, bool SERVER>
 __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
+    dependent_launch_prologue();
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
@@ -535,6 +556,7 @@ __device__ __forceinline__ void asgd_vectors(const AsgdArgs& a, const unsigned l
 
 template <bool DET, int NL>
 __global__ void asgd_kernel(const __grid_constant__ AsgdArgs a) {
+    dependent_launch_prologue();
     const unsigned long long nvec = a.n / NL;
     const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;

@@ -55,6 +55,27 @@ def test_reference_arm_prints_one_line_from_rank_zero():
     assert d["vs_baseline"] is None and d["higher_is_better"] is True
 
 
+def test_plain_start_with_gpus_launches_the_ranks_itself():
+    """`python bench.py --gpus 2` without torchrun becomes the launcher of its two ranks."""
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="", OMP_NUM_THREADS="1")
+    for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        env.pop(k, None)
+    res = subprocess.run([sys.executable, "bench.py", "--impl", "reference", "--gpus", "2", "--steps", "2",
+                          "--warmup", "1", "--workload", "lenet5", "--cpu-sample", "100000"],
+                         cwd=ROOT, env=env, capture_output=True, text=True, timeout=240)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = _json_lines(res.stdout)
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["impl"] == "reference"
+    # the CUDA arm refuses, in words, to start more ranks than there are devices
+    res = subprocess.run([sys.executable, "bench.py", "--gpus", "2", "--steps", "2"], cwd=ROOT, env=env,
+                         capture_output=True, text=True, timeout=240)
+    assert res.returncode != 0 and "CUDA device" in res.stderr
+    import bench
+
+    cmd = bench.self_launch_command(["--gpus", "4", "--steps", "3"], 4, 29999)
+    assert "--nproc-per-node=4" in cmd and cmd[-4:] == ["--gpus", "4", "--steps", "3"] and "127.0.0.1" in cmd
+
+
 def test_single_process_aggregate_is_identity():
     from paper_2005_06728_b200 import benchutil
 
