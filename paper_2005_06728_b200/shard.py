@@ -1,0 +1,220 @@
+"""The exchange steps either side of the update pass when the server role is spread over R GPUs.
+
+In the paper a worker reduces its gradient inside the node, pushes it to the parameter server
+and pulls the new weights back (Section 2.2, Fig. 3); OD-SGD overlaps the push with the local
+update and the pull with the next iteration's broadcast and compute (Section 3.1; Algorithm 2,
+repeat-loop).  Every element of the server's update is independent of the others, so on a
+multi-GPU node the server role shards by index: rank r of R owns the slice of every arena that
+odsgd_shard_range gives it.  One iteration is then
+
+    push          every worker sends slice s of its gradient to rank s.  The owner ends up with
+                  N separate shard buffers in its own memory, one per worker, in worker order.
+                  This is an all-to-all, not a reduce-scatter: a reduction inside the collective
+                  would add the workers in the collective's order, and the server rule adds them
+                  in worker order 0..N-1 (which is what makes results reproducible bit for bit).
+    server step   the library's global-update (or SSGD) kernel on the shard, summing the N
+                  buffers in worker order: the same kernel, the same arithmetic, on a slice.
+    pull          all-gather of the updated slices into every rank's replica of the weights.
+    local update  meanwhile, on a second stream, each worker compensates the weights it already
+                  has with its own gradient (odsgd_worker_local_update); it reads only the
+                  gradient and the old replica, so it overlaps the push.
+
+Only torch.distributed collectives into this GPU's own memory are used (NCCL on GPUs, gloo on
+CPU tensors in the tests); no kernel is handed a peer's memory.  Nothing here computes an update:
+the arithmetic stays in the CUDA library; this module moves slices and orders streams.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+from . import binding
+
+
+@dataclass(frozen=True)
+class ShardLayout:
+    """How an arena of `n_params` elements is spread over `n_ranks` ranks, each hosting
+    `workers_per_rank` workers.  Worker ids are global: worker j of rank q is q * k + j."""
+
+    n_params: int
+    n_ranks: int
+    workers_per_rank: int = 1
+
+    @property
+    def n_workers(self) -> int:
+        return self.n_ranks * self.workers_per_rank
+
+    @property
+    def shard_len(self) -> int:
+        """Nominal slice length: ceil(n_params / n_ranks) rounded up to 4 elements, the same for
+        every rank (odsgd_shard_range cuts the same slices and clips them to n_params)."""
+        per = -(-self.n_params // self.n_ranks)
+        return -(-per // 4) * 4
+
+    @property
+    def padded_len(self) -> int:
+        """Length of the arenas the exchange works on: n_ranks equal slices (zero padding at the end)."""
+        return self.shard_len * self.n_ranks
+
+    def owned(self, rank: int) -> Tuple[int, int]:
+        """[begin, end) of the elements rank `rank` owns (odsgd_shard_range)."""
+        return binding.shard_range(self.n_params, self.n_ranks, rank)
+
+    def worker_id(self, rank: int, j: int) -> int:
+        return rank * self.workers_per_rank + j
+
+
+class ShardExchange:
+    """push / pull over a torch.distributed process group.  Works on tensors of any device the
+    group's backend supports (CUDA with NCCL; CPU with gloo, which is how the tests run it)."""
+
+    def __init__(self, layout: ShardLayout, rank: int, group=None):
+        import torch.distributed as dist
+
+        self.layout, self.rank, self.group, self._dist = layout, rank, group, dist
+        if dist.get_world_size(group) != layout.n_ranks:
+            raise ValueError(f"process group has {dist.get_world_size(group)} ranks, layout has {layout.n_ranks}")
+
+    def push(self, grads: Sequence[torch.Tensor], recv: Sequence[torch.Tensor]) -> None:
+        """grads[j]: worker j of this rank, `padded_len` elements.  recv[j] (same length) receives,
+        at [q * S, (q + 1) * S), slice `rank` of the gradient of worker j of rank q."""
+        for g, r in zip(grads, recv):
+            self._dist.all_to_all_single(r, g, group=self.group)
+
+    def pull(self, w_full: torch.Tensor) -> None:
+        """All-gather, in place: every rank contributes its own slice of `w_full`."""
+        S = self.layout.shard_len
+        self._dist.all_gather_into_tensor(w_full, w_full[self.rank * S:(self.rank + 1) * S], group=self.group)
+
+
+def shard_views(layout: ShardLayout, rank: int, recv: Sequence[torch.Tensor]) -> List[torch.Tensor]:
+    """The N per-worker shard buffers of rank `rank`, as views into its receive buffers, in worker
+    order m = q * k + j; each has the length of the slice the rank owns."""
+    S = layout.shard_len
+    b, e = layout.owned(rank)
+    own = e - b
+    return [recv[j][q * S:q * S + own] for q in range(layout.n_ranks) for j in range(layout.workers_per_rank)]
+
+
+class ShardedOdsgd:
+    """One rank of the sharded update: the server role on the slice it owns, the worker role for
+    the workers it hosts.  CUDA only (the kernels are the library's).
+
+    The three phases of an iteration are separate methods so that a test can run several
+    emulated ranks in lockstep on one device; `step` runs them in order with the real exchange.
+    """
+
+    def __init__(self, layout: ShardLayout, rank: int, w0: torch.Tensor, *, lr: float, local_lr: float,
+                 momentum: float, wd: float, exchange, device: Optional[torch.device] = None, flags: int = 0,
+                 local_rule: int = binding.LOCAL_SGD, rule_lambda: float = 0.0, rule_m: float = 0.0,
+                 rule_eps: float = 0.0, warmup: int = 0):
+        dev = w0.device if device is None else device
+        if dev.type != "cuda":
+            raise RuntimeError("ShardedOdsgd runs the CUDA library: it needs a CUDA device (there is no CPU path)")
+        if w0.numel() != layout.n_params:
+            raise ValueError(f"w0 has {w0.numel()} elements, layout has {layout.n_params}")
+        self.layout, self.rank, self.exchange, self.device = layout, rank, exchange, dev
+        n, k, N = layout.n_params, layout.workers_per_rank, layout.n_workers
+        L, S = layout.padded_len, layout.shard_len
+        self.w_full = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(2)]
+        self.w_full[0][:n].copy_(w0)
+        self.cur = 0
+        self.recv = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)]
+        self.local = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)]
+        self.begin, self.end = layout.owned(rank)
+        own = self.end - self.begin
+        self.warmup, self.iteration = int(warmup), 0
+        self.side = torch.cuda.Stream(device=dev)
+        self.local_done = torch.cuda.Event()
+        # server role: a context over the slices of the two weight replicas this rank owns
+        self.server = None
+        self.v = torch.zeros(max(own, 4), dtype=torch.float32, device=dev)
+        if own > 0:
+            b, e = self.begin, self.end
+            self.server = binding.Odsgd(self.w_full[0][b:e], self.v[:own], n_workers=N, lr=lr, local_lr=local_lr,
+                                        momentum=momentum, wd=wd, w_b=self.w_full[1][b:e], flags=flags)
+            self.shard_grads = self.server.bind_grads(shard_views(layout, rank, self.recv))
+        # worker role: a worker-only context over the whole arena
+        slots: List[Optional[torch.Tensor]] = [None] * N
+        for j in range(k):
+            slots[layout.worker_id(rank, j)] = self.local[j][:n]
+        self.worker = binding.Odsgd(self.w_full[0][:n], None, n_workers=N, lr=lr, local_lr=local_lr,
+                                    momentum=momentum, wd=wd, w_b=self.w_full[1][:n], local=slots,
+                                    flags=flags | binding.FLAG_WORKER_ONLY)
+        self.state = None
+        if local_rule != binding.LOCAL_SGD:
+            tab = None
+            if local_rule in (binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM):
+                self.state = [torch.zeros(n, dtype=torch.float32, device=dev) for _ in range(k)]
+                tab = [None] * N
+                for j in range(k):
+                    tab[layout.worker_id(rank, j)] = self.state[j]
+            self.worker.set_local_rule(local_rule, rule_lambda, rule_m, rule_eps, tab)
+
+    # -- queries
+    def weights(self) -> torch.Tensor:
+        """This rank's replica of the current global weights (valid once the pull has completed)."""
+        return self.w_full[self.cur][:self.layout.n_params]
+
+    def train_weights(self, j: int) -> torch.Tensor:
+        """What hosted worker j computes its next gradient on (Algorithm 2): the global weights
+        while the next iteration index is <= warmup, its local weights afterwards."""
+        if self.iteration <= self.warmup:
+            return self.weights()
+        return self.local[j][:self.layout.n_params]
+
+    def set_lr(self, lr: float) -> None:
+        if self.server is not None:
+            self.server.set_lr(lr)
+
+    def set_local_lr(self, local_lr: float) -> None:
+        self.worker.set_local_lr(local_lr)
+
+    # -- the phases of one iteration
+    def phase_local_and_push(self, grads: Sequence[torch.Tensor]) -> None:
+        """grads[j]: gradient of hosted worker j, `padded_len` elements on this device (zeros
+        beyond n_params).  Starts the local updates on the side stream and pushes the slices."""
+        lay, n = self.layout, self.layout.n_params
+        if len(grads) != lay.workers_per_rank or any(g.numel() != lay.padded_len for g in grads):
+            raise ValueError(f"need {lay.workers_per_rank} gradients of {lay.padded_len} elements")
+        self._delayed = self.iteration >= self.warmup
+        if self._delayed:
+            main = torch.cuda.current_stream(self.device)
+            self.side.wait_stream(main)  # the gradients and the replica are ready
+            for j, g in enumerate(grads):
+                self.worker.worker_local_update(lay.worker_id(self.rank, j), self.w_full[self.cur][:n], g[:n],
+                                                no_delay=self.iteration == self.warmup, stream=self.side)
+            self.local_done.record(self.side)
+        self.exchange.push(grads, self.recv)
+
+    def phase_server(self) -> None:
+        """The server rule on the slice this rank owns, over the N received shard buffers."""
+        if self.server is None:
+            return
+        if self._delayed:
+            self.server.global_update(self.shard_grads)  # reads replica `cur`, writes replica `cur ^ 1`
+        else:
+            self.server.ssgd_step(self.shard_grads)      # warm-up: in place
+
+    def phase_pull(self) -> None:
+        """All-gather of the updated slices; afterwards the replica holds the new global weights."""
+        if self._delayed:
+            self.cur ^= 1
+        self.exchange.pull(self.w_full[self.cur])
+        if self._delayed:
+            # the next iteration's local update reads the replica the pull just filled and writes
+            # the local arenas: both are ordered behind this iteration's local updates
+            torch.cuda.current_stream(self.device).wait_stream(self.side)
+        self.iteration += 1
+
+    def step(self, grads: Sequence[torch.Tensor]) -> None:
+        self.phase_local_and_push(grads)
+        self.phase_server()
+        self.phase_pull()
+
+    def close(self) -> None:
+        if self.server is not None:
+            self.server.close()
+        self.worker.close()
