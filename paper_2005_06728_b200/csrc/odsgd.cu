@@ -253,10 +253,21 @@ int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry
 
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
 int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry) {
-    // few workers: the pass is close to a copy and wants the shallow, wide shape
-    if constexpr (LOCAL != kLocalAll) {
-        if (a.n_workers <= kFewWorkers)
-            return launch_server_k<DET, NL, LOCAL, RULE, MULT, kFewBatch, kFewUnroll>(c, a, st, dry);
+    // the shape follows the worker count on the 128-bit path; the scalar fallback and the
+    // all-workers variants (whose shape is fixed inside the kernel) keep a single instantiation
+    if constexpr (LOCAL != kLocalAll && NL == 4) {
+        switch (server_shape_for(a.n_workers)) {
+            case kShape2x4: return launch_server_k<DET, NL, LOCAL, RULE, MULT, 2, 4>(c, a, st, dry);
+            case kShape3x4:
+                // 3 x 4 fits the register budget only without a state arena or a multiplier
+                // lookup in the tile; the variants that have one take 4 x 3 (no spills)
+                if constexpr (!MULT && !needs_state(RULE))
+                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, 3, 4>(c, a, st, dry);
+                else
+                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, 4, 3>(c, a, st, dry);
+            case kShape4x3: return launch_server_k<DET, NL, LOCAL, RULE, MULT, 4, 3>(c, a, st, dry);
+            default: break;
+        }
     }
     return launch_server_k<DET, NL, LOCAL, RULE, MULT, kBatch, kUnroll>(c, a, st, dry);
 }
@@ -269,12 +280,15 @@ int launch_server_t(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t s
 
 template <bool DET, int NL, int LOCAL>
 int launch_server_r(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t st, bool dry) {
-    if (LOCAL == kLocalNone) return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
-    switch (c->local_rule) {
-        case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
-        case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, mult, st, dry);
-        case ODSGD_LOCAL_MOMENTUM: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_MOMENTUM>(c, a, mult, st, dry);
-        default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, mult, st, dry);
+    if constexpr (LOCAL == kLocalNone) {
+        return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
+    } else {
+        switch (c->local_rule) {
+            case ODSGD_LOCAL_SGD: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
+            case ODSGD_LOCAL_DC_C: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_C>(c, a, mult, st, dry);
+            case ODSGD_LOCAL_MOMENTUM: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_MOMENTUM>(c, a, mult, st, dry);
+            default: return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_DC_A>(c, a, mult, st, dry);
+        }
     }
 }
 

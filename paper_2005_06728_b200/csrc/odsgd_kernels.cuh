@@ -37,22 +37,12 @@ namespace odsgd {
 // ------------------------------------------------------------------ tuning constants
 // Each can be overridden with -D for a sweep; the defaults are what measured best on B200.
 
-// Server kernel, general case: gradient loads per batch x vectors per thread.
+// Server kernel, many workers: gradient loads per batch x vectors per thread.
 #ifndef ODSGD_BATCH
 #define ODSGD_BATCH 8
 #endif
 #ifndef ODSGD_UNROLL
 #define ODSGD_UNROLL 2
-#endif
-// Server kernel with at most ODSGD_FEW_WORKERS workers (the pass is close to a 1:1 copy).
-#ifndef ODSGD_FEW_WORKERS
-#define ODSGD_FEW_WORKERS 4
-#endif
-#ifndef ODSGD_FEW_BATCH
-#define ODSGD_FEW_BATCH 2
-#endif
-#ifndef ODSGD_FEW_UNROLL
-#define ODSGD_FEW_UNROLL 4
 #endif
 // Server kernel with every worker's local update in the pass: plain rule / Eq. 4, Eq. 5-6.
 #ifndef ODSGD_ALLSGD_BATCH
@@ -67,36 +57,47 @@ namespace odsgd {
 #ifndef ODSGD_ALLDC_UNROLL
 #define ODSGD_ALLDC_UNROLL 1
 #endif
+// 1: one worker's Eq. 4 update in the pass: its previous local weights are fetched with the
+// weights at the top of the tile instead of after the gradient sum (+1.2 % measured).  Not done
+// for the rules with a state arena: two more vectors per tile pushed the kernel into spills
+// (Eq. 5-6: -3 %).  Issuing worker m + 1's loads ahead of worker m's stores in the all-workers
+// variants (a software pipeline over the workers) was measured too and lost 1-3 %.
+#ifndef ODSGD_ONE_DC_EARLY
+#define ODSGD_ONE_DC_EARLY 1
+#endif
 // Local and ASGD kernels: vectors per thread per tile.
 #ifndef ODSGD_SMALL_UNROLL
 #define ODSGD_SMALL_UNROLL 4
 #endif
-// Gradient loads: 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching.
+// Gradient loads: 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching,
+// 3 read-only path without L1 allocation and a 256-byte L2 prefetch hint, 4 read-only path without
+// L1 allocation under an L2 evict-first policy.
 #ifndef ODSGD_GRAD_LOAD
 #define ODSGD_GRAD_LOAD 1
 #endif
-// Stores: 0 streaming (st.global.cs), 1 default caching.
+// Stores: 0 streaming (st.global.cs), 1 default caching, 2 under an L2 evict-first policy.
 #ifndef ODSGD_STORE
 #define ODSGD_STORE 0
 #endif
-// > 0: __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS) on the server kernel (register cap).
+// Register cap of the server kernel: __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS).  512 x 1
+// allows 128 registers per thread, i.e. two resident CTAs of the default 256 threads; without
+// the cap the Eq. 5-6 instantiations take 131-141 registers and lose the second CTA (measured:
+// 4.6 instead of 6.9 TB/s).  Launches wider than ODSGD_MAX_BLOCK threads are refused by the host.
 #ifndef ODSGD_MIN_CTAS
-#define ODSGD_MIN_CTAS 0
+#define ODSGD_MIN_CTAS 1
 #endif
 #ifndef ODSGD_MAX_BLOCK
-#define ODSGD_MAX_BLOCK 256
+#define ODSGD_MAX_BLOCK 512
 #endif
 
 constexpr int kBatch = ODSGD_BATCH;
 constexpr int kUnroll = ODSGD_UNROLL;
-constexpr int kFewWorkers = ODSGD_FEW_WORKERS;
-constexpr int kFewBatch = ODSGD_FEW_BATCH;
-constexpr int kFewUnroll = ODSGD_FEW_UNROLL;
 constexpr int kAllSgdBatch = ODSGD_ALLSGD_BATCH;
 constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
 constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
 constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
+constexpr bool kOneDcEarly = ODSGD_ONE_DC_EARLY != 0;
 #if ODSGD_MIN_CTAS > 0
 #define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
 #else
@@ -113,6 +114,21 @@ constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels
 constexpr int kServerCtasPerSm = 64;
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
+
+// Launch shape of the server kernel by worker count M: gradient loads per batch x vectors per
+// thread.  A batch that M divides evenly leaves no half-empty round of loads, and the fewer the
+// streams, the more vectors per thread it takes to keep enough bytes in flight.  Measured on
+// the 138 M-parameter arena (GB/s of algorithmic bytes, fused update), best shape per M:
+//   M <= 2: 2 x 4        M = 3, 5, 6, 9: 3 x 4        M = 4, 7, 8, 10..16: 4 x 3        M > 16: 8 x 2
+// (3 x 4 against 8 x 2: +3 % at M = 3, +4 % at M = 5 and 9; 4 x 3 against 8 x 2: +2 % at M = 12;
+// 8 x 2 wins from M = 24 on; 4 x 4, 6 x 3 and 2 x 6 spill registers and lose 15-25 %.)
+enum ServerShape : int { kShape2x4 = 0, kShape3x4 = 1, kShape4x3 = 2, kShapeMany = 3 };
+__host__ __device__ constexpr int server_shape_for(int n_workers) {
+    return n_workers <= 2 ? kShape2x4
+           : (n_workers == 3 || n_workers == 5 || n_workers == 6 || n_workers == 9) ? kShape3x4
+           : n_workers <= 16 ? kShape4x3
+                             : kShapeMany;
+}
 
 // Vectors per thread per tile of the server kernel: UB as instantiated, except when the pass
 // also carries every worker's local update (fewer when that update is delay-compensated and
@@ -206,12 +222,28 @@ __device__ __forceinline__ Vec<1> load_stream<1>(const float* p) {
 // that reads them, so they may also go through the read-only path.
 template <int NL>
 __device__ __forceinline__ Vec<NL> load_grad(const float* p);
+#if ODSGD_GRAD_LOAD == 4 || ODSGD_STORE == 2
+__device__ __forceinline__ unsigned long long evict_first_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+#endif
+
 template <>
 __device__ __forceinline__ Vec<4> load_grad<4>(const float* p) {
 #if ODSGD_GRAD_LOAD == 1
     const float4 t = __ldg(reinterpret_cast<const float4*>(p));
 #elif ODSGD_GRAD_LOAD == 2
     const float4 t = *reinterpret_cast<const float4*>(p);
+#elif ODSGD_GRAD_LOAD == 3
+    float4 t;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "l"(p));
+#elif ODSGD_GRAD_LOAD == 4
+    float4 t;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "l"(p), "l"(evict_first_policy()));
 #else
     const float4 t = __ldcs(reinterpret_cast<const float4*>(p));
 #endif
@@ -234,6 +266,9 @@ template <>
 __device__ __forceinline__ void store_stream<4>(float* p, const Vec<4>& a) {
 #if ODSGD_STORE == 1
     *reinterpret_cast<float4*>(p) = make_float4(a.e[0], a.e[1], a.e[2], a.e[3]);
+#elif ODSGD_STORE == 2
+    asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 :: "l"(p), "f"(a.e[0]), "f"(a.e[1]), "f"(a.e[2]), "f"(a.e[3]), "l"(evict_first_policy()) : "memory");
 #else
     __stcs(reinterpret_cast<float4*>(p), make_float4(a.e[0], a.e[1], a.e[2], a.e[3]));
 #endif
@@ -332,11 +367,19 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                                                const bool (&ok)[U], TensorCursor& cur) {
     using O = Op<DET>;
     Vec<NL> w[U], v[U], s[U], gl[U];
+    // one worker's Eq. 4 rule: its previous local weights are fetched early (only with two vectors
+    // per thread or fewer: the wide few-worker shape has no registers to spare)
+    constexpr bool kOneDc = LOCAL == kLocalOne && needs_prev(RULE) && !needs_state(RULE) && kOneDcEarly && U <= 2;
+    Vec<NL> xe[kOneDc ? U : 1], mse[kOneDc ? U : 1];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (ok[u]) {
             w[u] = load_stream<NL>(a.w_in + off[u]);
             v[u] = load_stream<NL>(a.v + off[u]);
+            if (kOneDc) {
+                if (needs_prev(RULE)) xe[u] = a.lp.first ? w[u] : load_stream<NL>(a.x[0] + off[u]);
+                if (needs_state(RULE)) mse[u] = load_stream<NL>(a.ms[0] + off[u]);
+            }
         }
     }
     // With every worker's delay-compensated local update in the pass, the previous local weights
@@ -423,8 +466,13 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
         if (LOCAL == kLocalOne) {
             float* xp = a.x[0];
             Vec<NL> xo, xv, msv;
-            if (needs_prev(RULE)) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
-            if (needs_state(RULE)) msv = load_stream<NL>(a.ms[0] + off[u]);
+            if (kOneDc) {
+                xv = xe[u];
+                msv = mse[u];
+            } else {
+                if (needs_prev(RULE)) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+                if (needs_state(RULE)) msv = load_stream<NL>(a.ms[0] + off[u]);
+            }
 #pragma unroll
             for (int l = 0; l < NL; ++l) {
                 xo.e[l] = local_rule<DET, RULE>(w[u].e[l], gl[u].e[l], xv.e[l], msv.e[l], a.lp);
@@ -438,9 +486,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
     }
 }
 
-// BB x UB: gradient loads per batch x vectors per thread.  8 x 2 for many workers; with four
-// workers or fewer the kernel is close to a copy and 2 x 4 (fewer registers, more resident
-// warps, more vectors per thread) measured 7-20 % faster.
+// BB x UB: gradient loads per batch x vectors per thread (server_shape_for picks them).
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ ServerArgs a) {
     dependent_launch_prologue();
