@@ -94,6 +94,9 @@ def parse_args(argv=None):
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra-kernels", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the other parameter sets (only the headline workload)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="spread the server role over the N ranks (all-to-all of gradient slices, update of the owned "
+                         "slice, all-gather of the weights) instead of N independent replicas")
     ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="elements in the reference arm's sample")
     return ap.parse_args(argv)
 
@@ -619,6 +622,100 @@ def run_cuda(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- sharded server arm
+def run_sharded(args):
+    """One OD-SGD iteration per step with the server role sharded over the ranks: every rank hosts
+    M / N workers, pushes the slices of their gradients to the owners, updates the slice it owns
+    and gathers the new weights, while the hosted workers' local updates run on a second stream.
+    Total work is fixed as N grows (strong scaling)."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2005_06728_b200 import binding, shard
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import ClockSampler, aggregate, barrier, init_process_group, rank_info
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the update pass has no CPU path")
+    binding.load_library()
+    ri = rank_info()
+    world, rank = ri["world_size"], ri["rank"]
+    dev = torch.device("cuda", ri["local_rank"])
+    torch.cuda.set_device(dev)
+    if world > 1:
+        init_process_group("nccl")
+    elif not dist.is_initialized():
+        import socket
+
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    wl = W.workload(args.workload)
+    M = args.workers or wl.n_workers
+    if M % world:
+        raise SystemExit(f"--sharded: {M} workers do not divide over {world} ranks")
+    k = M // world
+    n = wl.arena_len
+    lay = shard.ShardLayout(n, world, k)
+    w0 = W.make_weights(wl, dev)
+    sh = shard.ShardedOdsgd(lay, rank, w0, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                            exchange=shard.ShardExchange(lay, rank),
+                            flags=binding.FLAG_ALLOW_FMA if args.allow_fma else 0)
+    sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
+    grads = []
+    for j in range(k):
+        g = torch.zeros(lay.padded_len, dtype=torch.float32, device=dev)
+        W.make_grad(wl, lay.worker_id(rank, j), 0, dev, out=g[:n], _sigma=sg, _pads=pads)
+        grads.append(g)
+    stream = torch.cuda.current_stream()
+    for _ in range(max(3, args.warmup)):
+        sh.step(grads)
+    torch.cuda.synchronize()
+    barrier(dev)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(dev.index or 0) as clocks:
+        a.record(stream)
+        for _ in range(args.steps):
+            sh.step(grads)
+        b.record(stream)
+        torch.cuda.synchronize()
+    barrier(dev)
+    torch.cuda.synchronize()
+    P = wl.n_params
+    own = sh.end - sh.begin
+    # bytes this rank's kernels move per step: server rule on its slice, local rule for its k workers
+    local_bytes = (M + 4) * 4 * own + k * 3 * 4 * P
+    agg = aggregate(a.elapsed_time(b), float(local_bytes) * args.steps, dev)
+    if rank != 0:
+        return 0
+    S = lay.shard_len
+    ck = clocks.summary()
+    value = agg["units"] / (agg["ms"] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": agg["ms"] / args.steps, "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{wl.name}-shaped parameter set, M={M} workers, sharded server + local updates",
+                   "n_params": P, "n_workers": M, "workers_per_rank": k, "shard_len": S,
+                   "bytes_per_step": (M + 4) * 4 * P + M * 3 * 4 * P,
+                   "exchange_bytes_per_rank_per_step": {"push_sent": k * (world - 1) * S * 4,
+                                                        "pull_received": (world - 1) * S * 4},
+                   "parallelism": f"server role sharded over {world} rank(s): all-to-all of gradient slices, "
+                                  "kernel on the owned slice, all-gather of the weights; local updates on a second stream",
+                   "note": "value counts the bytes the update kernels move (server rule on every slice + every worker's "
+                           "local rule), not the bytes on the links"},
+        "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),
+                   "samples": ck.get("samples"), "source": ck.get("source")},
+        "e2e": None, "gpu_launches": args.steps * (k + (1 if own > 0 else 0)),
+        "params_per_s": P * args.steps / (agg["ms"] * 1e-3),
+    }
+    print(json.dumps(line), flush=True)
+    sh.close()
+    return 0
+
+
 # ----------------------------------------------------------------------------- launching N ranks
 def self_launch_command(argv, n_gpus, port):
     """The torchrun command line that runs this script as `n_gpus` ranks on this node."""
@@ -650,7 +747,7 @@ def main(argv=None):
     if args.impl == "reference":
         return run_reference(args)
     try:
-        return run_cuda(args)
+        return run_sharded(args) if args.sharded else run_cuda(args)
     finally:
         try:
             import torch.distributed as dist
