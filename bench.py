@@ -50,14 +50,14 @@ def hbm_peak():
 
 
 def measured_traffic(step_bytes):
-    """DRAM bytes per launch from the committed ncu capture of the fused kernel, scaled by the
-    algorithmic bytes (traffic grows in proportion: every stream is touched once).  None when the
+    """DRAM bytes per launch from the committed ncu capture of the fused kernel (the M = 32
+    instantiation on a smaller arena), scaled by the algorithmic bytes (traffic grows in proportion: every stream is touched once).  None when the
     kernel source has changed since the counters were taken."""
     import hashlib
     import re
 
     try:
-        note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_alexnet_m8.md")).read()
+        note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_m32_resnet50_arena.md")).read()
         src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
         ratio = float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1))
         sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1)

@@ -5,18 +5,20 @@
 //   * every input stream is read exactly once and every output written once;
 //   * 128-bit loads and stores, each warp touching 512 contiguous bytes per
 //     stream per instruction, each CTA walking contiguous tiles of every stream;
-//   * the M gradient streams are fetched in batches of kBatch x kUnroll
-//     independent 128-bit loads per thread before the dependent adds start
-//     (about 160 KB in flight per SM at two resident CTAs); the adds themselves
-//     stay in worker order 0..M-1; with few workers, or with every worker's
-//     local update fused in, shallower batches and more resident warps win;
+//   * the M gradient streams are fetched in batches of B x U independent
+//     128-bit loads per thread (B workers x U vectors) before the dependent adds
+//     start: 8 x 2 with many workers (about 160 KB in flight per SM at two
+//     resident CTAs), shapes with a batch that divides the worker count and more
+//     vectors per thread when there are few (server_shape_for); the adds
+//     themselves stay in worker order 0..M-1; with every worker's local update
+//     fused in, shallower batches and more resident warps win;
 //   * gradients go through the read-only path (ld.global.nc), which measured
 //     5-8 % faster here than streaming loads (ld.global.cs); state that is read
 //     and written by the same kernel uses coherent loads; results are stored
 //     with the streaming policy;
 //   * a grid of SMs x 64 CTAs at most strides over the tiles, so one launch
 //     covers the whole arena whatever the number of tensors in it, and the
-//     hardware scheduler evens out the tail.
+//     hardware scheduler evens out the tail;
 //   * every kernel opens with the two programmatic-dependent-launch instructions: it lets the
 //     next kernel of the stream be scheduled at once (griddepcontrol.launch_dependents) and
 //     itself waits, before its first memory access, until the kernels ahead of it have
