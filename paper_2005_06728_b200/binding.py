@@ -180,6 +180,13 @@ class BoundGrads:
             self.ctx._check(self.ctx._lib.odsgd_unbind_grads(self.ctx._h, self.slot))
             self.slot = -1
 
+    def __del__(self):
+        try:  # give the slot back when the table is dropped while its context is still alive
+            if self.slot >= 0 and self.ctx._h:
+                self.ctx._lib.odsgd_unbind_grads(self.ctx._h, self.slot)
+        except Exception:
+            pass
+
     def __len__(self) -> int:
         return len(self.tensors)
 
