@@ -334,7 +334,51 @@ def _sweep(s, worker_counts, reps, stream, peak):
     return rows
 
 
-def _small_set_entry(name, dev, stream, flags, steps=4000, graph_steps=20):
+def _end_to_end(s, step_bytes, steps, stream, dev, world=1):
+    """The fused update through the host-buffer entry point: every step copies the M gradients
+    from pinned host memory, runs the kernel and copies the worker's new weights back, all
+    inside the timed region.  The set's gradient arenas serve as the device staging buffers."""
+    import torch
+
+    from paper_2005_06728_b200 import workloads as W
+    from paper_2005_06728_b200.benchutil import aggregate, barrier
+
+    wl, M, ctx, n = s.wl, s.M, s.ctx, s.wl.arena_len
+    pool = [W.make_grad(wl, m, 1, dev, _sigma=s.sg, _pads=s.pads).cpu().pin_memory() for m in range(min(M, 4))]
+    host_grads = [pool[m % len(pool)] for m in range(M)]
+    host_out = torch.empty(n, dtype=torch.float32).pin_memory()
+    # copy-back on a second stream overlaps the next step's uploads; for small arenas the
+    # cross-stream hand-over costs more than it hides, so they keep a single stream
+    copy_stream = torch.cuda.Stream(device=dev) if n * 4 >= (1 << 26) else None
+    ctx.fused_update_host(host_grads, s.grads, 0, host_out, stream, copy_stream)
+    torch.cuda.synchronize()
+    barrier(dev)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    a.record(stream)
+    for _ in range(steps):
+        ctx.fused_update_host(host_grads, s.grads, 0, host_out, stream, copy_stream)
+    if copy_stream is not None:
+        stream.wait_stream(copy_stream)  # the last copy-back is inside the timed region
+    b.record(stream)
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - t0) * 1e3
+    e2e_ms = max(a.elapsed_time(b), wall_ms)
+    agg2 = aggregate(e2e_ms, float(step_bytes) * steps, dev if world > 1 else None)
+    h2d, d2h = M * n * 4, n * 4
+    return {"value": agg2["units"] / (agg2["ms"] * 1e-3) / 1e9, "unit": "GB/s",
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
+            "ms_per_step": agg2["ms"] / steps,
+            "h2d_GBps": h2d * steps * world / (agg2["ms"] * 1e-3) / 1e9,
+            "what": "ALGORITHMIC bytes of the update, (M + 5) * 4 * P per step, over a time that is set by the "
+                    "host link: M * 4 * P bytes cross it per step (h2d_GBps is that traffic over the same time), "
+                    "so this figure may sit above what the bus itself carries",
+            "note": f"{M} host-to-device copies per step from a pool of {len(pool)} distinct pinned buffers; "
+                    + ("copy-back of the local weights on a second stream" if copy_stream is not None
+                       else "copy-back on the same stream (small arena)")}
+
+
+def _small_set_entry(name, dev, stream, flags, cpu_full=True, steps=4000, graph_steps=20):
     """A cache-resident set: eager launches through the bound-table call, and CUDA-graph replay."""
     import torch
 
@@ -372,11 +416,13 @@ def _small_set_entry(name, dev, stream, flags, steps=4000, graph_steps=20):
     for k, r in rules.items():
         if k != "fused":
             entry[k] = {"us": r["ms"] * 1e3, "effective_GBps": r["GBps"], "frac": None}
+    if cpu_full:
+        entry["cpu_oracle_full"] = time_oracle_full(wl, wl.n_workers, s.w_a, s.grads, passes=5)
     ctx.close()
     return entry
 
 
-def _large_set_entry(name, dev, stream, flags, peak, reps, cpu_full):
+def _large_set_entry(name, dev, stream, flags, peak, reps, cpu_full, e2e):
     import torch
 
     from paper_2005_06728_b200 import workloads as W
@@ -390,6 +436,8 @@ def _large_set_entry(name, dev, stream, flags, peak, reps, cpu_full):
     entry.update(_all_rules(s, reps, stream, peak))
     entry["params_per_s"] = wl.n_params / (entry["fused"]["ms"] * 1e-3)
     entry["grad_elems_per_s"] = wl.n_workers * entry["params_per_s"]
+    if e2e:
+        entry["e2e"] = _end_to_end(s, entry["bytes_per_step"], 6, stream, dev)
     if cpu_full:
         entry["cpu_oracle_full"] = time_oracle_full(wl, wl.n_workers, s.w_a, s.grads)
     s.ctx.close()
@@ -535,40 +583,7 @@ def run_cuda(args):
     # ---- end to end: gradients start in pinned host memory, local weights come back
     e2e = None
     if not args.no_e2e:
-        pool = [W.make_grad(wl, m, 1, dev, _sigma=head.sg, _pads=head.pads).cpu().pin_memory() for m in range(min(M, 4))]
-        host_grads = [pool[m % len(pool)] for m in range(M)]
-        host_out = torch.empty(n, dtype=torch.float32).pin_memory()
-        e2e_steps = max(2, min(args.steps, 6))
-        # copy-back on a second stream overlaps the next step's uploads; for small arenas the
-        # cross-stream hand-over costs more than it hides, so they keep a single stream
-        copy_stream = torch.cuda.Stream(device=dev) if n * 4 >= (1 << 26) else None
-        ctx.fused_update_host(host_grads, grad_list, 0, host_out, stream, copy_stream)
-        torch.cuda.synchronize()
-        barrier(dev)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t0 = time.perf_counter()
-        a.record(stream)
-        for _ in range(e2e_steps):
-            ctx.fused_update_host(host_grads, grad_list, 0, host_out, stream, copy_stream)
-        if copy_stream is not None:
-            stream.wait_stream(copy_stream)  # the last copy-back is inside the timed region
-        b.record(stream)
-        torch.cuda.synchronize()
-        wall_ms = (time.perf_counter() - t0) * 1e3
-        e2e_ms = max(a.elapsed_time(b), wall_ms)
-        agg2 = aggregate(e2e_ms, float(step_bytes) * e2e_steps, dev if world > 1 else None)
-        h2d, d2h = M * n * 4, n * 4
-        e2e = {"value": agg2["units"] / (agg2["ms"] * 1e-3) / 1e9, "unit": "GB/s",
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-               "ms_per_step": agg2["ms"] / e2e_steps,
-               "h2d_GBps": h2d * e2e_steps * world / (agg2["ms"] * 1e-3) / 1e9,
-               "what": "ALGORITHMIC bytes of the update, (M + 5) * 4 * P per step, over a time that is set by the "
-                       "host link: M * 4 * P bytes cross it per step (h2d_GBps is that traffic over the same time), "
-                       "so this figure may sit above what the bus itself carries",
-               "note": f"{M} host-to-device copies per step from a pool of {len(pool)} distinct pinned buffers; "
-                       + ("copy-back of the local weights on a second stream" if copy_stream is not None
-                          else "copy-back on the same stream (small arena)")}
-        del pool, host_grads, host_out
+        e2e = _end_to_end(head, step_bytes, max(2, min(args.steps, 6)), stream, dev, world)
 
     if not rank0:
         return 0
@@ -588,9 +603,9 @@ def run_cuda(args):
         torch.cuda.empty_cache()
         for name in ("alexnet", "resnet50"):
             configs.append(_large_set_entry(name, dev, stream, flags, peak, reps=200,
-                                            cpu_full=not args.no_cpu_baseline))
+                                            cpu_full=not args.no_cpu_baseline, e2e=not args.no_e2e))
         for name in ("resnet56", "lenet5"):
-            configs.append(_small_set_entry(name, dev, stream, flags))
+            configs.append(_small_set_entry(name, dev, stream, flags, cpu_full=not args.no_cpu_baseline))
 
     ck = clocks.summary()
     roof_frac = achieved / peak if hbm_bound else None

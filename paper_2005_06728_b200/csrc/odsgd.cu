@@ -246,7 +246,7 @@ int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry
     auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT, BB, UB>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     if (dry) return ODSGD_OK;
-    const int grid = grid_for(c, a.n, NL, block, server_vectors_per_thread(LOCAL, RULE, UB), kServerCtasPerSm);
+    const int grid = grid_for(c, a.n, NL, block, server_vectors_per_thread(LOCAL, RULE, UB), server_grid_cap(a.n_workers));
     launch_kernel<ServerArgs>(kernel, grid, block, st, a);
     return after_launch(c, "server kernel launch");
 }
@@ -312,10 +312,10 @@ int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, 
 
 template <bool DET, int NL, int RULE, bool SERVER>
 int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultLocalBlock;
     auto kernel = local_kernel<DET, NL, RULE, SERVER>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, st, a);
+    launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kLocalCtasPerSm), block, st, a);
     return after_launch(c, "local kernel launch");
 }
 
@@ -341,10 +341,10 @@ int launch_local(odsgd_ctx* c, const LocalArgs& a, int lanes, bool server, cudaS
 
 template <bool DET, int NL>
 int launch_asgd_t(odsgd_ctx* c, const AsgdArgs& a, cudaStream_t st) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultSmallBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : kDefaultAsgdBlock;
     auto kernel = asgd_kernel<DET, NL>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    launch_kernel<AsgdArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kServerCtasPerSm), block, st, a);
+    launch_kernel<AsgdArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kAsgdCtasPerSm), block, st, a);
     return after_launch(c, "asgd kernel launch");
 }
 

@@ -16,9 +16,10 @@
 //     5-8 % faster here than streaming loads (ld.global.cs); state that is read
 //     and written by the same kernel uses coherent loads; results are stored
 //     with the streaming policy;
-//   * a grid of SMs x 64 CTAs at most strides over the tiles, so one launch
-//     covers the whole arena whatever the number of tensors in it, and the
-//     hardware scheduler evens out the tail;
+//   * one launch covers the whole arena whatever the number of tensors in it: a
+//     grid capped per SM (server_grid_cap) strides over the tiles, close to one
+//     tile per CTA when tiles are heavy so that the hardware scheduler evens out
+//     the tail, close to persistent for the copy-like one-worker pass;
 //   * every kernel opens with the two programmatic-dependent-launch instructions: it lets the
 //     next kernel of the stream be scheduled at once (griddepcontrol.launch_dependents) and
 //     itself waits, before its first memory access, until the kernels ahead of it have
@@ -109,11 +110,19 @@ constexpr bool kOneDcEarly = ODSGD_ONE_DC_EARLY != 0;
 // Launch shape (used by the host side; kept here so that everything that decides how the
 // kernels touch memory lives in one file).
 constexpr int kDefaultBlock = 256;       // server kernel
-constexpr int kDefaultSmallBlock = 512;  // local and ASGD kernels
-// Grid cap in CTAs per SM.  More CTAs than can be resident (two at the server kernel's
-// register count) measured 1-2 % faster than an exactly persistent grid: late SMs pick up
-// the remaining tiles.
-constexpr int kServerCtasPerSm = 64;
+constexpr int kDefaultLocalBlock = 512;  // local kernel
+constexpr int kDefaultAsgdBlock = 256;   // ASGD kernel (256 against 512 threads: +0.6-1.4 % on the mid-size arenas)
+// Grid cap in CTAs per SM; the grid strides over the tiles beyond it.  How much a CTA should
+// loop depends on how heavy a tile is.  With many gradient streams a tile is hundreds of KB and
+// finer-grained scheduling evens out the tail: 256 per SM (in effect one tile per CTA) measured
+// 0.6-1.9 % faster than 64 from M = 4 up, and than an exactly persistent grid.  The copy-like
+// one-worker pass has light tiles and pays for CTA turnover instead: 16 per SM is 6 % faster
+// than 64 on the 25-61 M-parameter arenas (equal on the 138 M one); two workers sit in between.
+constexpr int kLocalCtasPerSm = 128;
+constexpr int kAsgdCtasPerSm = 256;
+__host__ __device__ constexpr int server_grid_cap(int n_workers) {
+    return n_workers <= 1 ? 16 : (n_workers == 2 ? 64 : 256);
+}
 
 enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
 
