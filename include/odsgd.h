@@ -309,7 +309,10 @@ int odsgd_set_local_rule(odsgd_ctx* ctx, int rule, float lambda, float m, float 
  * off.  Applies to the global, fused and SSGD calls; the ASGD and local rules are unaffected.
  * The 128-bit kernels need every tensor offset to be a multiple of 4 elements; otherwise the
  * call fails with ERR_ALIGN unless ODSGD_FLAG_ALLOW_UNALIGNED is set (scalar kernel).
- * Errors: ERR_CUDA (allocation or copy failed), ERR_ALIGN.
+ * Call it outside stream capture (ERR_STATE while `stream` is capturing: the call may allocate, and
+ * a captured upload would re-read the host copy of the table at every replay); update calls that
+ * use the table can be captured afterwards.
+ * Errors: ERR_CUDA (allocation or copy failed), ERR_ALIGN, ERR_STATE (wrong current device, capture).
  */
 int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const float* wd_mult, void* stream);
 

@@ -933,6 +933,15 @@ int odsgd_set_tensor_multipliers(odsgd_ctx* ctx, const float* lr_mult, const flo
     // the table is allocated, filled and freed on the context's own device
     const int rc_dev = on_own_device(c);
     if (rc_dev != ODSGD_OK) return rc_dev;
+    // not while `stream` is capturing: the call may allocate, and a captured upload would re-read
+    // the context's host copy of the table at every replay (whatever a later call left there)
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cap) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, ODSGD_ERR_CUDA, "cudaStreamIsCapturing failed");
+    }
+    if (cap != cudaStreamCaptureStatusNone)
+        return fail(c, ODSGD_ERR_STATE, "odsgd_set_tensor_multipliers cannot be recorded into a stream capture");
     if (!lr_mult && !wd_mult) {
         if (c->table_dev) cudaFree(c->table_dev);
         c->table_dev = nullptr;

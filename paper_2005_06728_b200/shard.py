@@ -172,6 +172,14 @@ class ShardedOdsgd:
     def set_local_lr(self, local_lr: float) -> None:
         self.worker.set_local_lr(local_lr)
 
+    def set_momentum(self, momentum: float) -> None:
+        if self.server is not None:
+            self.server.set_momentum(momentum)
+
+    def set_wd(self, wd: float) -> None:
+        if self.server is not None:
+            self.server.set_wd(wd)
+
     # -- the phases of one iteration
     def phase_local_and_push(self, grads: Sequence[torch.Tensor]) -> None:
         """grads[j]: gradient of hosted worker j, `padded_len` elements on this device (zeros

@@ -232,6 +232,29 @@ def test_pending_copy_back_is_respected_by_every_stream(cuda_device):
     assert torch.equal(local[1], lr_[1]) and torch.equal(ctx.weights(), ref.weights())
 
 
+def test_multiplier_setter_refuses_stream_capture(cuda_device):
+    """The table upload (and a possible allocation) does not belong in a graph; update calls that
+    use a table set beforehand can be captured."""
+    wl = W.ragged_workload([4_096, 4_096], n_workers=2)
+    a, _, va, la = _ctx(wl, (0,))
+    b, _, vb, lb = _ctx(wl, (0,))
+    grads = W.make_grads(wl, 0, DEV)
+    for c in (a, b):
+        c.set_tensor_multipliers([1.0, 0.5], [1.0, 0.0])
+        c.fused_update(grads, 0), c.fused_update(grads, 0)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        with pytest.raises(binding.OdsgdError) as e:
+            a.set_tensor_multipliers([2.0, 2.0], None)
+        a.fused_update(grads, 0), a.fused_update(grads, 0)
+    assert e.value.code == binding.ERR_STATE
+    graph.replay()
+    b.fused_update(grads, 0), b.fused_update(grads, 0)
+    torch.cuda.synchronize()
+    assert torch.equal(a.weights(), b.weights()) and torch.equal(va, vb) and torch.equal(la[0], lb[0])
+
+
 def test_other_device_is_refused_without_a_launch(cuda_device):
     """With a second device current, every launching or allocating call answers ERR_STATE."""
     if torch.cuda.device_count() < 2:
