@@ -109,7 +109,7 @@ class ShardedOdsgd:
     def __init__(self, layout: ShardLayout, rank: int, w0: torch.Tensor, *, lr: float, local_lr: float,
                  momentum: float, wd: float, exchange, device: Optional[torch.device] = None, flags: int = 0,
                  local_rule: int = binding.LOCAL_SGD, rule_lambda: float = 0.0, rule_m: float = 0.0,
-                 rule_eps: float = 0.0, warmup: int = 0):
+                 rule_eps: float = 0.0, warmup: int = 0, tensor_offsets: Optional[Sequence[int]] = None):
         dev = w0.device if device is None else device
         if dev.type != "cuda":
             raise RuntimeError("ShardedOdsgd runs the CUDA library: it needs a CUDA device (there is no CPU path)")
@@ -131,10 +131,18 @@ class ShardedOdsgd:
         # server role: a context over the slices of the two weight replicas this rank owns
         self.server = None
         self.v = torch.zeros(max(own, 4), dtype=torch.float32, device=dev)
+        # the tensors (or parts of tensors) that fall into the owned slice, as offsets relative to it
+        offs = list(tensor_offsets) if tensor_offsets is not None else [0, n]
+        if offs[0] != 0 or offs[-1] != n:
+            raise ValueError("tensor_offsets must start at 0 and end at n_params")
+        self.slice_tensors = [t for t in range(len(offs) - 1) if offs[t] < self.end and offs[t + 1] > self.begin]
+        self.slice_offsets = [max(offs[t], self.begin) - self.begin for t in self.slice_tensors] + [own]
+        self.n_tensors = len(offs) - 1
         if own > 0:
             b, e = self.begin, self.end
             self.server = binding.Odsgd(self.w_full[0][b:e], self.v[:own], n_workers=N, lr=lr, local_lr=local_lr,
-                                        momentum=momentum, wd=wd, w_b=self.w_full[1][b:e], flags=flags)
+                                        momentum=momentum, wd=wd, w_b=self.w_full[1][b:e], flags=flags,
+                                        tensor_offsets=self.slice_offsets)
             self.shard_grads = self.server.bind_grads(shard_views(layout, rank, self.recv))
         # worker role: a worker-only context over the whole arena
         slots: List[Optional[torch.Tensor]] = [None] * N
@@ -171,6 +179,20 @@ class ShardedOdsgd:
 
     def set_local_lr(self, local_lr: float) -> None:
         self.worker.set_local_lr(local_lr)
+
+    def set_tensor_multipliers(self, lr_mult: Optional[Sequence[float]], wd_mult: Optional[Sequence[float]]) -> None:
+        """Per-tensor multipliers of the whole parameter set (one entry per tensor of
+        `tensor_offsets`); each rank keeps the entries of the tensors its slice touches."""
+        if self.server is None:
+            return
+        if lr_mult is None and wd_mult is None:
+            self.server.set_tensor_multipliers(None, None)
+            return
+        for m in (lr_mult, wd_mult):
+            if m is not None and len(m) != self.n_tensors:
+                raise ValueError(f"need {self.n_tensors} multipliers, got {len(m)}")
+        pick = lambda m: None if m is None else [float(m[t]) for t in self.slice_tensors]
+        self.server.set_tensor_multipliers(pick(lr_mult), pick(wd_mult))
 
     def set_momentum(self, momentum: float) -> None:
         if self.server is not None:

@@ -159,6 +159,55 @@ def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, ru
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("R", [1, 3, 8])
+def test_emulated_ranks_with_per_tensor_multipliers(cuda_device, R):
+    """Tensor boundaries cut by slice boundaries: each rank's server context gets the offsets and
+    multipliers of the (parts of) tensors in its slice, and the result equals the unsharded one."""
+    dev = torch.device("cuda:0")
+    wl = W.ragged_workload([1000, 12, 20_000, 4, 7_777, 3], n_workers=R, lr=0.1, local_lr=0.05, momentum=0.9, wd=1e-2)
+    n = wl.arena_len
+    lay = shard.ShardLayout(n, R, 1)
+    rng = np.random.default_rng(R)
+    lr_mult = rng.choice([0.0, 0.5, 1.0, 2.0], wl.n_tensors).tolist()
+    wd_mult = rng.choice([0.0, 1.0], wl.n_tensors).tolist()
+    w0 = W.make_weights(wl, dev)
+    w, v = w0.clone(), torch.zeros(n, device=dev)
+    local = [torch.zeros(n, device=dev) for _ in range(R)]
+    ref = binding.Odsgd(w, v, n_workers=R, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                        w_b=torch.zeros(n, device=dev), local=local, tensor_offsets=wl.offsets)
+    ref.set_tensor_multipliers(lr_mult, wd_mult)
+    hub = _Loopback(lay)
+    ranks = [shard.ShardedOdsgd(lay, r, w0, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                                exchange=hub.port(r), tensor_offsets=wl.offsets) for r in range(R)]
+    for sh in ranks:
+        sh.set_tensor_multipliers(lr_mult, wd_mult)
+    assert sum(len(sh.slice_tensors) for sh in ranks) >= wl.n_tensors, "every tensor is owned by some rank"
+    for it in range(3):
+        grads = [W.make_grad(wl, m, it, dev) for m in range(R)]
+        padded = []
+        for g in grads:
+            p = torch.zeros(lay.padded_len, device=dev)
+            p[:n].copy_(g)
+            padded.append(p)
+        ref.step_update(grads)
+        for r, sh in enumerate(ranks):
+            sh.phase_local_and_push([padded[r]])
+        hub.deliver_push()
+        for sh in ranks:
+            sh.phase_server()
+        for sh in ranks:
+            sh.phase_pull()
+        hub.deliver_pull()
+        torch.cuda.synchronize()
+        for r, sh in enumerate(ranks):
+            assert torch.equal(sh.weights(), ref.weights()), f"rank {r}, iteration {it}"
+            assert torch.equal(sh.train_weights(0), ref.train_weights(r))
+    for sh in ranks:
+        sh.close()
+    ref.close()
+
+
+@pytest.mark.gpu
 def test_single_rank_process_group_runs_the_real_exchange(cuda_device):
     """World size 1 over NCCL: the real collectives (degenerate: one rank) inside ShardedOdsgd.step."""
     import torch.distributed as dist
