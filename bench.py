@@ -51,8 +51,9 @@ def hbm_peak():
 
 def measured_traffic(step_bytes):
     """DRAM bytes per launch from the committed ncu capture of the fused kernel (the M = 32
-    instantiation on a smaller arena), scaled by the algorithmic bytes (traffic grows in proportion: every stream is touched once).  None when the
-    kernel source has changed since the counters were taken."""
+    instantiation on a smaller arena), scaled by the algorithmic bytes (traffic grows in
+    proportion: every stream is touched once).  None when the kernel source has changed since
+    the counters were taken."""
     import hashlib
     import re
 
