@@ -577,7 +577,7 @@ def run_cuda(args):
 
     # ---- worker-count sweep on the same arena (fused update, first m gradient buffers)
     sweep_counts = [int(x) for x in args.sweep_workers.split(",") if x]
-    if not sweep_counts and not args.no_configs and args.workload == "vgg16" and not args.workers:
+    if not sweep_counts and not args.no_configs and world == 1 and args.workload == "vgg16" and not args.workers:
         sweep_counts = [1, 2, 4, 8, 16, 32]
     sweep = _sweep(head, sweep_counts, max(20, min(200, args.steps)), stream, peak) if sweep_counts and rank0 else []
 
