@@ -98,6 +98,9 @@ def parse_args(argv=None):
     ap.add_argument("--sharded", action="store_true",
                     help="spread the server role over the N ranks (all-to-all of gradient slices, update of the owned "
                          "slice, all-gather of the weights) instead of N independent replicas")
+    ap.add_argument("--peer", action="store_true",
+                    help="with --sharded: no collective on the data path; the server kernel reads the other ranks' "
+                         "gradient slices and writes their weight replicas through symmetric memory")
     ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="elements in the reference arm's sample")
     return ap.parse_args(argv)
 
@@ -680,13 +683,14 @@ def run_sharded(args):
     n = wl.arena_len
     lay = shard.ShardLayout(n, world, k)
     w0 = W.make_weights(wl, dev)
+    exchange = shard.PeerExchange(lay, rank, dev) if args.peer else shard.ShardExchange(lay, rank)
     sh = shard.ShardedOdsgd(lay, rank, w0, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
-                            exchange=shard.ShardExchange(lay, rank),
-                            flags=binding.FLAG_ALLOW_FMA if args.allow_fma else 0)
+                            exchange=exchange, flags=binding.FLAG_ALLOW_FMA if args.allow_fma else 0)
     sg, pads = W.sigma_arena(wl, dev), W.pad_mask(wl, dev)
     grads = []
     for j in range(k):
-        g = torch.zeros(lay.padded_len, dtype=torch.float32, device=dev)
+        # the peer exchange reads the gradients where the workers produce them: its own arenas
+        g = exchange.grad_arenas[j] if args.peer else torch.zeros(lay.padded_len, dtype=torch.float32, device=dev)
         W.make_grad(wl, lay.worker_id(rank, j), 0, dev, out=g[:n], _sigma=sg, _pads=pads)
         grads.append(g)
     stream = torch.cuda.current_stream()
@@ -723,8 +727,11 @@ def run_sharded(args):
                    "bytes_per_step": (M + 4) * 4 * P + M * 3 * 4 * P,
                    "exchange_bytes_per_rank_per_step": {"push_sent": k * (world - 1) * S * 4,
                                                         "pull_received": (world - 1) * S * 4},
-                   "parallelism": f"server role sharded over {world} rank(s): all-to-all of gradient slices, "
-                                  "kernel on the owned slice, all-gather of the weights; local updates on a second stream",
+                   "parallelism": (f"server role sharded over {world} rank(s): the kernel on the owned slice reads "
+                                   "the other ranks' gradient slices and writes their replicas through symmetric "
+                                   "memory, one fence either side; local updates on a second stream") if args.peer else
+                                  (f"server role sharded over {world} rank(s): all-to-all of gradient slices, "
+                                   "kernel on the owned slice, all-gather of the weights; local updates on a second stream"),
                    "note": "value counts the bytes the update kernels move (server rule on every slice + every worker's "
                            "local rule), not the bytes on the links"},
         "clocks": {"sm_mhz": ck.get("sm_mhz"), "sm_max_mhz": ck.get("sm_max_mhz"), "reasons": ck.get("reasons", []),

@@ -75,6 +75,9 @@ extern "C" {
 #define ODSGD_FLAG_ALLOW_FMA 0x4u       /* let multiply-add pairs fuse (excludes ODSGD_FLAG_DETERMINISTIC) */
 #define ODSGD_FLAG_WORKER_ONLY 0x8u     /* worker-role context: v may be NULL; only odsgd_worker_local_update runs */
 
+/* Largest number of weight mirrors per weight arena (odsgd_set_weight_mirrors). */
+#define ODSGD_MAX_MIRRORS 15
+
 /* Gradient tables one context can keep bound at a time (odsgd_bind_grads). */
 #define ODSGD_MAX_BINDINGS 16
 
@@ -263,6 +266,38 @@ int odsgd_worker_local_update(odsgd_ctx* ctx, int worker_id, const float* w_bak,
  * Host arithmetic only.  Errors: ERR_ARG (NULL output, n_ranks < 1, rank out of range).
  */
 int odsgd_shard_range(size_t n_params, int n_ranks, int rank, size_t* begin, size_t* end);
+
+/*
+ * Weight mirrors: further device buffers that receive every weight the server pass writes, by
+ * the kernel's own stores.  With the server role spread over R GPUs (odsgd_shard_range), each
+ * rank updates the slice it owns, and every rank needs the whole new vector before its workers
+ * can use it: Section 2.2's pull (Fig. 3), which Section 3.1 overlaps with the next iteration.
+ * A context over the owned slice whose mirrors are that same slice inside the other R - 1 ranks'
+ * replicas (their memory mapped into this process: CUDA IPC or symmetric memory, with peer
+ * access enabled) delivers the new weights while it computes them; no all-gather follows the
+ * kernel.  The same holds on the read side without any call: entries of `worker_grads` may be
+ * peer-mapped memory of another GPU, so that the push needs no staging copy.  The kernels touch
+ * all of these with ordinary 128-bit loads and stores only (no bulk-copy engine, no multicast).
+ *   mirrors_a, mirrors_b  HOST arrays of n_mirrors DEVICE pointers, n_params floats each:
+ *                         mirrors_a[i] shadows w_a, mirrors_b[i] shadows w_b (ping-pong layout:
+ *                         both tables; in-place layout: mirrors_b must be NULL).  A call that
+ *                         writes weight half h also writes h's mirrors, same offsets, same bits.
+ *   n_mirrors             0 .. ODSGD_MAX_MIRRORS; 0 switches the feature off (tables ignored).
+ * While mirrors are set only odsgd_global_update / odsgd_ssgd_step and their *_bound forms run
+ * (they carry no local update; workers use odsgd_worker_local_update on their own replica); the
+ * fused, scheduled, ASGD and DC-ASGD calls fail with ERR_STATE because they would leave the
+ * mirrors stale.  The library never reads a mirror and does not initialise it: the caller fills
+ * each with w_0.  Mirrors count as state buffers: they must not overlap one another, the
+ * context's arenas or a gradient buffer (ERR_OVERLAP, here or in the update call), and setting
+ * them invalidates bound gradient tables like any other change of the state buffers.  Ordering
+ * between GPUs is the caller's: the peers' gradients must be complete before the call's kernel
+ * starts, and a peer may read its replica only after that kernel has finished (for instance a
+ * stream-ordered collective on either side).  The library cannot tell a peer-mapped address
+ * from a local one and cannot check that peer access is enabled.
+ * Errors: ERR_ARG (NULL table or entry, count out of range, mirrors_b against the layout),
+ * ERR_ALIGN, ERR_OVERLAP, ERR_STATE (worker-only context).
+ */
+int odsgd_set_weight_mirrors(odsgd_ctx* ctx, float* const* mirrors_a, float* const* mirrors_b, int n_mirrors);
 
 /*
  * Hyper-parameters are kernel arguments, never compiled in: the paper's runs change the

@@ -23,6 +23,7 @@ FLAG_ALLOW_UNALIGNED = 0x2
 FLAG_ALLOW_FMA = 0x4
 FLAG_WORKER_ONLY = 0x8
 MAX_BINDINGS = 16
+MAX_MIRRORS = 15
 LOCAL_SGD, LOCAL_DC_C, LOCAL_DC_A, LOCAL_MOMENTUM = 0, 1, 2, 3
 
 OK, ERR_ARG, ERR_ALIGN, ERR_OVERLAP, ERR_STATE, ERR_CUDA, ERR_UNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
@@ -39,6 +40,7 @@ EXPORTS = (
     "odsgd_lr_poly_decay", "odsgd_fused_update_mult_static", "odsgd_get_iteration", "odsgd_set_iteration",
     "odsgd_bind_grads", "odsgd_unbind_grads", "odsgd_global_update_bound", "odsgd_fused_update_bound",
     "odsgd_ssgd_step_bound", "odsgd_step_bound", "odsgd_worker_local_update", "odsgd_shard_range",
+    "odsgd_set_weight_mirrors",
 )
 
 
@@ -118,6 +120,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
         "odsgd_worker_local_update": ([vp, ci, vp, vp, ci, vp], ci),
         "odsgd_shard_range": ([ctypes.c_size_t, ci, ci, ctypes.POINTER(ctypes.c_size_t),
                                ctypes.POINTER(ctypes.c_size_t)], ci),
+        "odsgd_set_weight_mirrors": ([vp, pvp, pvp, ci], ci),
     }
     for name, (argtypes, restype) in sig.items():
         fn = getattr(lib, name)  # AttributeError if the library lacks a declared symbol
@@ -400,6 +403,24 @@ class Odsgd:
         self._check(self._lib.odsgd_fused_update_mult_static(self._h, self._grad_table(grads), worker_id,
                                                              arr(lr_mult), arr(wd_mult), _stream_handle(stream)))
         self._bound = grads
+
+    def set_weight_mirrors(self, mirrors_a: Optional[Sequence[torch.Tensor]],
+                           mirrors_b: Optional[Sequence[torch.Tensor]] = None) -> None:
+        """odsgd_set_weight_mirrors: tensors (n_params elements each; local or peer-mapped memory)
+        that receive every weight the server pass writes into w_a (mirrors_a) / w_b (mirrors_b).
+        None or an empty list switches the feature off."""
+        if not mirrors_a:
+            self._check(self._lib.odsgd_set_weight_mirrors(self._h, None, None, 0))
+            self._mirrors = None
+            return
+        if mirrors_b is not None and len(mirrors_b) != len(mirrors_a):
+            raise ValueError("mirrors_a and mirrors_b need the same number of entries")
+        ta = _ptr_table([_dev_ptr(t, f"mirrors_a[{i}]", self.n_params) for i, t in enumerate(mirrors_a)])
+        tb = None
+        if mirrors_b is not None:
+            tb = _ptr_table([_dev_ptr(t, f"mirrors_b[{i}]", self.n_params) for i, t in enumerate(mirrors_b)])
+        self._check(self._lib.odsgd_set_weight_mirrors(self._h, ta, tb, len(mirrors_a)))
+        self._mirrors = (list(mirrors_a), list(mirrors_b) if mirrors_b is not None else None)
 
     def set_server_mean_square(self, ms: Optional[torch.Tensor]) -> None:
         self._check(self._lib.odsgd_set_server_mean_square(self._h, _dev_ptr(ms, "mean_square", self.n_params)))

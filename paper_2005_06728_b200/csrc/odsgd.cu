@@ -49,6 +49,9 @@ struct odsgd_ctx {
     std::vector<unsigned char> table_host;  // staging copy the upload reads from
     bool mult_on = false;
     float* server_ms = nullptr;  // Eq. 6 state of the server-side DC-ASGD step
+    // weight mirrors: mirror[h][i] receives what the server kernel writes into weight half h
+    float* mirror[2][ODSGD_MAX_MIRRORS] = {};
+    int n_mirrors = 0;
     uint64_t wp = 0;             // Algorithm 2's warm-up length
     uint64_t iter = 0;           // iterations done through odsgd_step
     // host-buffer entry point with a separate copy stream: ordering between the two streams
@@ -107,7 +110,7 @@ struct BufList {
         if (n < CAP) b[n++] = Named{p, name, idx};
     }
 };
-constexpr int kMaxState = 5 + 2 * ODSGD_MAX_WORKERS;
+constexpr int kMaxState = 5 + 2 * ODSGD_MAX_WORKERS + 2 * ODSGD_MAX_MIRRORS;
 using StateList = BufList<kMaxState>;
 using CallList = BufList<kMaxState + ODSGD_MAX_WORKERS + 4>;
 
@@ -123,6 +126,10 @@ void state_buffers(const odsgd_ctx* c, StateList* s) {
         if (c->mean_square[m]) s->add(c->mean_square[m], "mean_square", m);
     }
     if (c->server_ms) s->add(c->server_ms, "server_mean_square", -1);
+    for (int i = 0; i < c->n_mirrors; ++i) {
+        s->add(c->mirror[0][i], "mirrors_a", i);
+        if (c->mirror[1][i]) s->add(c->mirror[1][i], "mirrors_b", i);
+    }
 }
 
 int check_distinct(odsgd_ctx* err_ctx, const StateList& s, size_t bytes) {
@@ -280,7 +287,7 @@ int launch_server_t(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t s
 
 template <bool DET, int NL, int LOCAL>
 int launch_server_r(odsgd_ctx* c, const ServerArgs& a, bool mult, cudaStream_t st, bool dry) {
-    if constexpr (LOCAL == kLocalNone) {
+    if constexpr (LOCAL == kLocalNone || LOCAL == kLocalNoneMirrored) {
         return launch_server_t<DET, NL, LOCAL, ODSGD_LOCAL_SGD>(c, a, mult, st, dry);
     } else {
         switch (c->local_rule) {
@@ -297,6 +304,7 @@ int launch_server_l(odsgd_ctx* c, const ServerArgs& a, int local_mode, bool mult
     switch (local_mode) {
         case kLocalNone: return launch_server_r<DET, NL, kLocalNone>(c, a, mult, st, dry);
         case kLocalOne: return launch_server_r<DET, NL, kLocalOne>(c, a, mult, st, dry);
+        case kLocalNoneMirrored: return launch_server_r<DET, NL, kLocalNoneMirrored>(c, a, mult, st, dry);
         default: return launch_server_r<DET, NL, kLocalAll>(c, a, mult, st, dry);
     }
 }
@@ -492,6 +500,18 @@ int plan_server(odsgd_ctx* c, const float* const* grads, bool keep_backup, int l
     if (a.w_prev) ptrs.add(a.w_prev, "w_delayed", -1);
 
     p->local_mode = kLocalNone;
+    if (c->n_mirrors > 0) {
+        // only the plain server pass keeps mirrors in step with the weights
+        if (local_id >= -1)
+            return fail(c, ODSGD_ERR_STATE, "weight mirrors are set: only odsgd_global_update / odsgd_ssgd_step (and their bound forms) can run");
+        const int half = a.w_out == c->w[1] ? 1 : 0;
+        for (int i = 0; i < c->n_mirrors; ++i) {
+            a.w_mirror[i] = c->mirror[half][i];
+            ptrs.add(a.w_mirror[i], half ? "mirrors_b" : "mirrors_a", i);
+        }
+        a.n_mirrors = c->n_mirrors;
+        p->local_mode = kLocalNoneMirrored;
+    }
     if (local_id >= -1) {
         const int rc = bind_local_outputs(c, local_id, &a, &p->local_mode, &ptrs);
         if (rc != ODSGD_OK) return rc;
@@ -843,6 +863,7 @@ int odsgd_asgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stre
     if (worker_id < 0 || worker_id >= c->n_workers) return fail(c, ODSGD_ERR_ARG, "worker_id out of range");
     if (!grad) return fail(c, ODSGD_ERR_ARG, "grad is NULL");
     if (!c->v) return fail(c, ODSGD_ERR_STATE, "a worker-only context (ODSGD_FLAG_WORKER_ONLY) has no server state");
+    if (c->n_mirrors > 0) return fail(c, ODSGD_ERR_STATE, "weight mirrors are set: the ASGD step would leave them stale");
     StateList st;
     state_buffers(c, &st);
     const int rc_o = check_outside(c, st, Named{grad, "grad", -1});
@@ -999,6 +1020,46 @@ int odsgd_set_server_mean_square(odsgd_ctx* ctx, float* mean_square) {
     return ODSGD_OK;
 }
 
+int odsgd_set_weight_mirrors(odsgd_ctx* ctx, float* const* mirrors_a, float* const* mirrors_b, int n_mirrors) {
+    if (!ctx) return ODSGD_ERR_ARG;
+    odsgd_ctx* c = ctx;
+    if (n_mirrors < 0 || n_mirrors > ODSGD_MAX_MIRRORS)
+        return fail(c, ODSGD_ERR_ARG, "n_mirrors must be in 0.." + std::to_string(ODSGD_MAX_MIRRORS));
+    if (n_mirrors == 0) {
+        if (c->n_mirrors != 0) c->state_epoch += 1;
+        c->n_mirrors = 0;
+        return ODSGD_OK;
+    }
+    if (!c->v) return fail(c, ODSGD_ERR_STATE, "a worker-only context (ODSGD_FLAG_WORKER_ONLY) has no server pass to mirror");
+    if (!mirrors_a) return fail(c, ODSGD_ERR_ARG, "mirrors_a is NULL");
+    if (c->pingpong && !mirrors_b) return fail(c, ODSGD_ERR_ARG, "the ping-pong layout needs mirrors_b as well");
+    if (!c->pingpong && mirrors_b) return fail(c, ODSGD_ERR_ARG, "mirrors_b must be NULL in the in-place layout");
+    const size_t need = (c->flags & ODSGD_FLAG_ALLOW_UNALIGNED) ? 4 : 16;
+    for (int i = 0; i < n_mirrors; ++i) {
+        if (!mirrors_a[i] || (mirrors_b && !mirrors_b[i])) return fail(c, ODSGD_ERR_ARG, "NULL entry in a mirror table");
+        if (!aligned(mirrors_a[i], need) || (mirrors_b && !aligned(mirrors_b[i], need)))
+            return fail(c, ODSGD_ERR_ALIGN, "mirror " + std::to_string(i) + " is not " + std::to_string(need) + "-byte aligned");
+    }
+    float* keep[2][ODSGD_MAX_MIRRORS];
+    memcpy(keep, c->mirror, sizeof keep);
+    const int keep_n = c->n_mirrors;
+    for (int i = 0; i < ODSGD_MAX_MIRRORS; ++i) {
+        c->mirror[0][i] = i < n_mirrors ? mirrors_a[i] : nullptr;
+        c->mirror[1][i] = i < n_mirrors && mirrors_b ? mirrors_b[i] : nullptr;
+    }
+    c->n_mirrors = n_mirrors;
+    StateList st;
+    state_buffers(c, &st);
+    const int rc = check_distinct(c, st, c->n * sizeof(float));
+    if (rc != ODSGD_OK) {
+        memcpy(c->mirror, keep, sizeof keep);
+        c->n_mirrors = keep_n;
+        return rc;
+    }
+    c->state_epoch += 1;  // bound gradient tables were checked against the old set of buffers
+    return ODSGD_OK;
+}
+
 int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* stream) {
     if (!ctx) return ODSGD_ERR_ARG;
     odsgd_ctx* c = ctx;
@@ -1009,6 +1070,7 @@ int odsgd_dcasgd_step(odsgd_ctx* ctx, int worker_id, const float* grad, void* st
     if (!c->local[worker_id]) return fail(c, ODSGD_ERR_ARG, "no backup (local) buffer for worker " + std::to_string(worker_id));
     const bool need_ms = c->local_rule == ODSGD_LOCAL_DC_A;
     if (need_ms && !c->server_ms) return fail(c, ODSGD_ERR_STATE, "ODSGD_LOCAL_DC_A at the server needs odsgd_set_server_mean_square");
+    if (c->n_mirrors > 0) return fail(c, ODSGD_ERR_STATE, "weight mirrors are set: the DC-ASGD step would leave them stale");
     StateList st;
     state_buffers(c, &st);
     const int rc_o = check_outside(c, st, Named{grad, "grad", -1});

@@ -124,7 +124,11 @@ __host__ __device__ constexpr int server_grid_cap(int n_workers) {
     return n_workers <= 1 ? 16 : (n_workers == 2 ? 64 : 256);
 }
 
-enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2 };
+// What else the server pass carries: nothing, one worker's local update, every worker's, or -
+// with no local update - a copy of the new weights into each of the context's weight mirrors
+// (the other ranks' replicas when the server role is sharded: the pull of Section 2.2 done by
+// the kernel's own stores instead of a collective behind it).
+enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2, kLocalNoneMirrored = 3 };
 
 // Launch shape of the server kernel by worker count M: gradient loads per batch x vectors per
 // thread.  A batch that M divides evenly leaves no half-empty round of loads, and the fewer the
@@ -168,6 +172,8 @@ struct ServerArgs {
     float* w_out;                       // weights after the update (may equal w_in)
     float* w_prev;                      // optional copy of the old weights
     float* v;                           // momentum state, in place
+    float* w_mirror[ODSGD_MAX_MIRRORS]; // kLocalNoneMirrored: further destinations of the new weights
+    int n_mirrors;
     unsigned long long n;               // elements
     int n_workers;
     int local_worker;                   // kLocalOne: whose gradient feeds x[0]
@@ -494,6 +500,11 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
         if (a.w_prev != nullptr) store_stream<NL>(a.w_prev + off[u], w[u]);
         store_stream<NL>(a.v + off[u], vn);
         store_stream<NL>(a.w_out + off[u], wn);
+        if (LOCAL == kLocalNoneMirrored) {
+            // the same vector to every mirror (plain stores: a mirror may be peer-mapped memory
+            // of another GPU, reached over NVLink)
+            for (int r = 0; r < a.n_mirrors; ++r) store_stream<NL>(a.w_mirror[r] + off[u], wn);
+        }
     }
 }
 

@@ -19,9 +19,24 @@ odsgd_shard_range gives it.  One iteration is then
                   has with its own gradient (odsgd_worker_local_update); it reads only the
                   gradient and the old replica, so it overlaps the push.
 
-Only torch.distributed collectives into this GPU's own memory are used (NCCL on GPUs, gloo on
-CPU tensors in the tests); no kernel is handed a peer's memory.  Nothing here computes an update:
-the arithmetic stays in the CUDA library; this module moves slices and orders streams.
+Two ways to move the slices:
+
+    ShardExchange   torch.distributed collectives into this GPU's own memory (NCCL on GPUs, gloo
+                    on CPU tensors in the tests): all-to-all before the kernel, all-gather after.
+    PeerExchange    no collective on the data path.  Gradient arenas and weight replicas live in
+                    symmetric memory, so every rank has every other rank's buffers mapped.  The
+                    server kernel reads the N gradient slices where they are (its own workers'
+                    locally, the others' over NVLink) and stores each new weight into the owned
+                    slice of all R replicas (odsgd_set_weight_mirrors): push, update and pull are
+                    one pass, the transfers overlap the arithmetic element by element, and the
+                    staging copies of the all-to-all (one extra write and read of N slices per
+                    rank) disappear.  Plain 128-bit loads and stores only: no bulk-copy engine and
+                    no multicast touch a peer's memory.  What remains between ranks is ordering: a
+                    stream-ordered fence before the kernel (every rank's gradients are complete)
+                    and one after it (every rank's slice has landed in this replica).
+
+Nothing here computes an update: the arithmetic stays in the CUDA library; this module moves
+slices, maps buffers and orders streams.
 """
 from __future__ import annotations
 
@@ -89,6 +104,59 @@ class ShardExchange:
         self._dist.all_gather_into_tensor(w_full, w_full[self.rank * S:(self.rank + 1) * S], group=self.group)
 
 
+class PeerExchange:
+    """Buffers of the sharded update in symmetric memory, and the fences between ranks.
+
+    One symmetric allocation per rank holds its k gradient arenas and its two weight replicas
+    (`padded_len` floats each); after the rendezvous every rank can address every other rank's
+    copy of it.  The caller writes worker j's gradient into `grad_arenas[j]`; ShardedOdsgd takes
+    the replicas, the gradient table of its server kernel (`peer_grad`) and the mirrors of its
+    weight stores (`peer_replica`) from here.  `fence()` is a one-element all-reduce on the
+    current stream: it completes on a rank only once every rank has reached it in stream order,
+    which is all the ordering the kernels need (they never wait on one another themselves).
+    """
+
+    direct = True
+
+    def __init__(self, layout: ShardLayout, rank: int, device: torch.device, group=None):
+        import os
+
+        import torch.distributed as dist
+
+        # nothing here uses the NVSwitch multicast mapping symmetric memory would otherwise set up
+        os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")
+        import torch.distributed._symmetric_memory as symm_mem
+
+        if dist.get_world_size(group) != layout.n_ranks:
+            raise ValueError(f"process group has {dist.get_world_size(group)} ranks, layout has {layout.n_ranks}")
+        if layout.n_ranks - 1 > binding.MAX_MIRRORS:
+            raise ValueError(f"at most {binding.MAX_MIRRORS + 1} ranks (one weight mirror per other rank)")
+        self.layout, self.rank, self.group, self._dist = layout, rank, group, dist
+        k, L = layout.workers_per_rank, layout.padded_len
+        self._total = (k + 2) * L
+        self._own = symm_mem.empty(self._total, dtype=torch.float32, device=device)
+        self._own.zero_()
+        self._hdl = symm_mem.rendezvous(self._own, dist.group.WORLD if group is None else group)
+        self._whole = [self._own if q == rank else self._hdl.get_buffer(q, (self._total,), torch.float32)
+                       for q in range(layout.n_ranks)]
+        self._token = torch.zeros(1, dtype=torch.float32, device=device)
+        self.grad_arenas = [self.peer_grad(rank, j) for j in range(k)]
+        self.replicas = [self.peer_replica(rank, h) for h in range(2)]
+
+    def peer_grad(self, q: int, j: int) -> torch.Tensor:
+        """Gradient arena of worker j of rank q, as mapped into this process."""
+        L = self.layout.padded_len
+        return self._whole[q][j * L:(j + 1) * L]
+
+    def peer_replica(self, q: int, half: int) -> torch.Tensor:
+        """Weight replica `half` (0 / 1) of rank q, as mapped into this process."""
+        k, L = self.layout.workers_per_rank, self.layout.padded_len
+        return self._whole[q][(k + half) * L:(k + half + 1) * L]
+
+    def fence(self) -> None:
+        self._dist.all_reduce(self._token, group=self.group)
+
+
 def shard_views(layout: ShardLayout, rank: int, recv: Sequence[torch.Tensor]) -> List[torch.Tensor]:
     """The N per-worker shard buffers of rank `rank`, as views into its receive buffers, in worker
     order m = q * k + j; each has the length of the slice the rank owns."""
@@ -104,6 +172,13 @@ class ShardedOdsgd:
 
     The three phases of an iteration are separate methods so that a test can run several
     emulated ranks in lockstep on one device; `step` runs them in order with the real exchange.
+
+    `exchange` is a ShardExchange (collectives around the kernel) or anything with
+    `direct = True` and PeerExchange's members (`replicas`, `grad_arenas`, `peer_grad`,
+    `peer_replica`, `fence`): then the server kernel itself reads the peers' gradient slices and
+    writes the peers' replicas, the gradients passed to `phase_local_and_push` must be the
+    exchange's own `grad_arenas`, and `w0` has to be the same on every rank (each fills its own
+    replicas with it).
     """
 
     def __init__(self, layout: ShardLayout, rank: int, w0: torch.Tensor, *, lr: float, local_lr: float,
@@ -118,10 +193,18 @@ class ShardedOdsgd:
         self.layout, self.rank, self.exchange, self.device = layout, rank, exchange, dev
         n, k, N = layout.n_params, layout.workers_per_rank, layout.n_workers
         L, S = layout.padded_len, layout.shard_len
-        self.w_full = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(2)]
-        self.w_full[0][:n].copy_(w0)
+        self.direct = bool(getattr(exchange, "direct", False))
+        if self.direct:
+            self.w_full = list(exchange.replicas)
+            for h in range(2):  # the mirrors are never read, but a replica is: both start as w_0
+                self.w_full[h].zero_()
+                self.w_full[h][:n].copy_(w0)
+            self.recv = []
+        else:
+            self.w_full = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(2)]
+            self.w_full[0][:n].copy_(w0)
+            self.recv = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)]
         self.cur = 0
-        self.recv = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)]
         self.local = [torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)]
         self.begin, self.end = layout.owned(rank)
         own = self.end - self.begin
@@ -143,7 +226,17 @@ class ShardedOdsgd:
             self.server = binding.Odsgd(self.w_full[0][b:e], self.v[:own], n_workers=N, lr=lr, local_lr=local_lr,
                                         momentum=momentum, wd=wd, w_b=self.w_full[1][b:e], flags=flags,
                                         tensor_offsets=self.slice_offsets)
-            self.shard_grads = self.server.bind_grads(shard_views(layout, rank, self.recv))
+            if self.direct:
+                R = layout.n_ranks
+                others = [q for q in range(R) if q != rank]
+                if others:
+                    self.server.set_weight_mirrors([exchange.peer_replica(q, 0)[b:e] for q in others],
+                                                   [exchange.peer_replica(q, 1)[b:e] for q in others])
+                # the N gradient slices where they are, in worker order m = q * k + j
+                self.shard_grads = self.server.bind_grads(
+                    [exchange.peer_grad(q, j)[b:e] for q in range(R) for j in range(k)])
+            else:
+                self.shard_grads = self.server.bind_grads(shard_views(layout, rank, self.recv))
         # worker role: a worker-only context over the whole arena
         slots: List[Optional[torch.Tensor]] = [None] * N
         for j in range(k):
@@ -217,7 +310,14 @@ class ShardedOdsgd:
                 self.worker.worker_local_update(lay.worker_id(self.rank, j), self.w_full[self.cur][:n], g[:n],
                                                 no_delay=self.iteration == self.warmup, stream=self.side)
             self.local_done.record(self.side)
-        self.exchange.push(grads, self.recv)
+        if self.direct:
+            if any(g.data_ptr() != a.data_ptr() for g, a in zip(grads, self.exchange.grad_arenas)):
+                raise ValueError("with a direct exchange the gradients must be written into exchange.grad_arenas")
+            # every rank's gradients are complete, and every rank is done with the replica half
+            # and the gradient arenas of the previous iteration, before any server kernel starts
+            self.exchange.fence()
+        else:
+            self.exchange.push(grads, self.recv)
 
     def phase_server(self) -> None:
         """The server rule on the slice this rank owns, over the N received shard buffers."""
@@ -232,7 +332,10 @@ class ShardedOdsgd:
         """All-gather of the updated slices; afterwards the replica holds the new global weights."""
         if self._delayed:
             self.cur ^= 1
-        self.exchange.pull(self.w_full[self.cur])
+        if self.direct:
+            self.exchange.fence()  # every rank's kernel has finished: all slices of the replica are in
+        else:
+            self.exchange.pull(self.w_full[self.cur])
         if self._delayed:
             # the next iteration's local update reads the replica the pull just filled and writes
             # the local arenas: both are ordered behind this iteration's local updates

@@ -4,7 +4,8 @@ On CPU (world size 2 and 3 over gloo): the package's push / pull move the right 
 right owners in worker order, and an update applied slice by slice between them gathers to
 exactly what the oracle computes on the whole arena.  On one GPU: R emulated ranks of
 ShardedOdsgd, driven phase by phase through an in-process stand-in for the collectives,
-reproduce the unsharded library bit for bit."""
+reproduce the unsharded library bit for bit - with the slices moved around the kernel, and with
+the kernel itself reading the other ranks' gradient arenas and writing their replicas."""
 import json
 import os
 import socket
@@ -104,10 +105,51 @@ class _Loopback:
                     self.pulled[dst][src * S:(src + 1) * S].copy_(piece)
 
 
+class _PeerHub:
+    """Stands in for symmetric memory when several ranks are emulated in one process: every rank's
+    gradient arenas and replicas are ordinary tensors of this device, and a "peer's" buffer is
+    simply the other emulated rank's tensor.  The ranks run in lockstep on one stream, so the
+    fences have nothing to do."""
+
+    def __init__(self, layout, dev):
+        k, L, R = layout.workers_per_rank, layout.padded_len, layout.n_ranks
+        self.layout = layout
+        self.grads = [[torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(k)] for _ in range(R)]
+        self.reps = [[torch.zeros(L, dtype=torch.float32, device=dev) for _ in range(2)] for _ in range(R)]
+        self.fences = 0
+
+    def port(self, rank):
+        hub = self
+
+        class Port:
+            direct = True
+            grad_arenas = hub.grads[rank]
+            replicas = hub.reps[rank]
+
+            def peer_grad(self, q, j):
+                return hub.grads[q][j]
+
+            def peer_replica(self, q, half):
+                return hub.reps[q][half]
+
+            def fence(self):
+                hub.fences += 1
+
+        return Port()
+
+    # the collectives of the other exchange have no counterpart here
+    def deliver_push(self):
+        pass
+
+    def deliver_pull(self):
+        pass
+
+
 @pytest.mark.gpu
 @pytest.mark.parametrize("R,k,n", [(2, 1, 100_003), (3, 2, 50_001), (8, 1, 200_000), (8, 2, 37), (2, 4, 8)])
 @pytest.mark.parametrize("rule", ["sgd", "dc_c"])
-def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, rule):
+@pytest.mark.parametrize("exchange", ["collectives", "direct"])
+def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, rule, exchange):
     dev = torch.device("cuda:0")
     lay = shard.ShardLayout(n, R, k)
     N, L = lay.n_workers, lay.padded_len
@@ -122,7 +164,8 @@ def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, ru
                         w_b=torch.zeros(n, device=dev), local=local)
     ref.set_local_rule(lrule, 0.04)
     ref.set_warmup(warmup)
-    hub = _Loopback(lay)
+    direct = exchange == "direct"
+    hub = _PeerHub(lay, dev) if direct else _Loopback(lay)
     ranks = [shard.ShardedOdsgd(lay, r, w0, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
                                 exchange=hub.port(r), local_rule=lrule, rule_lambda=0.04, warmup=warmup)
              for r in range(R)]
@@ -130,7 +173,8 @@ def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, ru
         grads = [W.make_grad(wl, m, it, dev)[:n] for m in range(N)]
         padded = []
         for m in range(N):
-            g = torch.zeros(L, device=dev)
+            # direct exchange: the gradient is produced in the arena the other ranks have mapped
+            g = hub.grads[m // k][m % k] if direct else torch.zeros(L, device=dev)
             g[:n].copy_(grads[m])
             padded.append(g)
         ref.step_update(grads)
@@ -153,6 +197,13 @@ def test_emulated_ranks_reproduce_the_unsharded_library(cuda_device, R, k, n, ru
                 m = lay.worker_id(r, j)
                 want = ref.train_weights(m)
                 assert torch.equal(sh.train_weights(j), want), f"train weights of worker {m}, iteration {it}"
+        if direct:
+            assert hub.fences == 2 * R * (it + 1), "one fence before and one after the server kernel, per rank"
+            for r in range(R):
+                assert all(bool(torch.all(g[n:] == 0)) for g in hub.grads[r]), "gradient padding untouched"
+    if direct:
+        with pytest.raises(ValueError, match="grad_arenas"):
+            ranks[0].phase_local_and_push([torch.zeros(L, device=dev) for _ in range(k)])
     for sh in ranks:
         sh.close()
     ref.close()
@@ -238,6 +289,53 @@ def test_single_rank_process_group_runs_the_real_exchange(cuda_device):
                 padded.append(p)
             ref.step_update(grads)
             sh.step(padded)
+            torch.cuda.synchronize()
+            assert torch.equal(sh.weights(), ref.weights()) and torch.equal(sh.v[:n], v)
+            for j in range(3):
+                assert torch.equal(sh.train_weights(j), ref.train_weights(j))
+        sh.close()
+        ref.close()
+    finally:
+        if created:
+            dist.destroy_process_group()
+
+
+@pytest.mark.gpu
+def test_single_rank_symmetric_memory_runs_the_direct_exchange(cuda_device):
+    """World size 1: PeerExchange's real symmetric-memory allocation, rendezvous, views and fences
+    inside ShardedOdsgd.step (degenerate: no other rank to map, no mirror)."""
+    import torch.distributed as dist
+
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    created = False
+    if not dist.is_initialized():
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{_free_port()}", rank=0, world_size=1)
+        created = True
+    try:
+        n = 300_001
+        lay = shard.ShardLayout(n, 1, 3)
+        wl = W.ragged_workload([n], n_workers=3, lr=0.1, local_lr=0.05, momentum=0.9, wd=1e-3, seed=9)
+        w0 = W.make_weights(wl, dev)[:n].clone()
+        w, v = w0.clone(), torch.zeros(n, device=dev)
+        local = [torch.zeros(n, device=dev) for _ in range(3)]
+        ref = binding.Odsgd(w, v, n_workers=3, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                            w_b=torch.zeros(n, device=dev), local=local)
+        ref.set_warmup(1)
+        ex = shard.PeerExchange(lay, 0, dev)
+        assert len(ex.grad_arenas) == 3 and all(g.numel() == lay.padded_len for g in ex.grad_arenas)
+        assert ex.peer_grad(0, 2).data_ptr() == ex.grad_arenas[2].data_ptr()
+        assert ex.peer_replica(0, 1).data_ptr() == ex.replicas[1].data_ptr()
+        assert all(g.data_ptr() % 16 == 0 for g in ex.grad_arenas + ex.replicas)
+        sh = shard.ShardedOdsgd(lay, 0, w0, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                                exchange=ex, warmup=1)
+        assert sh.w_full[0].data_ptr() == ex.replicas[0].data_ptr()
+        for it in range(4):
+            grads = [W.make_grad(wl, m, it, dev)[:n] for m in range(3)]
+            for a, g in zip(ex.grad_arenas, grads):
+                a[:n].copy_(g)
+            ref.step_update(grads)
+            sh.step(ex.grad_arenas)
             torch.cuda.synchronize()
             assert torch.equal(sh.weights(), ref.weights()) and torch.equal(sh.v[:n], v)
             for j in range(3):
