@@ -713,6 +713,8 @@ def run_sharded(args):
     # bytes this rank's kernels move per step: server rule on its slice, local rule for its k workers
     local_bytes = (M + 4) * 4 * own + k * 3 * 4 * P
     agg = aggregate(a.elapsed_time(b), float(local_bytes) * args.steps, dev)
+    if args.peer:
+        exchange.quiesce()  # no rank drops its symmetric buffers while a peer may still touch them
     if rank != 0:
         return 0
     S = lay.shard_len

@@ -249,7 +249,7 @@ int too_wide(odsgd_ctx* c, int block) {
 // kernel's register use), so that a caller can validate everything before it enqueues copies.
 template <bool DET, int NL, int LOCAL, int RULE, bool MULT, int BB, int UB>
 int launch_server_k(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : server_default_block(LOCAL, RULE);
     auto kernel = server_kernel<DET, NL, LOCAL, RULE, MULT, BB, UB>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     if (dry) return ODSGD_OK;

@@ -11,7 +11,7 @@
 //     resident CTAs), shapes with a batch that divides the worker count and more
 //     vectors per thread when there are few (server_shape_for); the adds
 //     themselves stay in worker order 0..M-1; with every worker's local update
-//     fused in, shallower batches and more resident warps win;
+//     fused in, shallower batches win (each worker's result leaves at once);
 //   * gradients go through the read-only path (ld.global.nc), which measured
 //     5-8 % faster here than streaming loads (ld.global.cs); state that is read
 //     and written by the same kernel uses coherent loads; results are stored
@@ -47,18 +47,31 @@ namespace odsgd {
 #ifndef ODSGD_UNROLL
 #define ODSGD_UNROLL 2
 #endif
-// Server kernel with every worker's local update in the pass: plain rule / Eq. 4, Eq. 5-6.
+// Server kernel with every worker's local update in the pass.  Each worker's result is stored as
+// soon as its gradient is in, so few workers per round of loads and more vectors per thread do
+// best: plain rule 2 x 4 (against 8 x 2: +2 % at M = 32, +4 % at M = 4, +13 % at M = 2 on the
+// 138 M-parameter arena, equal on the others; 3 x 4 and 2 x 5 tie, 1 x 4, 1 x 6, 2 x 6 lose 3-8 %);
+// Eq. 4: one worker per round, 2 vectors, 128-thread CTAs (+2 % over 1 vector x 256 threads; 3
+// vectors lose 4 %); Eq. 5-6 and local momentum: one worker, one vector, 128-thread CTAs (+2 %
+// for Eq. 5-6; two workers per round lose 15-20 %, two vectors 3-10 %).
 #ifndef ODSGD_ALLSGD_BATCH
-#define ODSGD_ALLSGD_BATCH ODSGD_BATCH
+#define ODSGD_ALLSGD_BATCH 2
 #endif
 #ifndef ODSGD_ALLSGD_UNROLL
-#define ODSGD_ALLSGD_UNROLL ODSGD_UNROLL
+#define ODSGD_ALLSGD_UNROLL 4
 #endif
 #ifndef ODSGD_ALLDC_BATCH
 #define ODSGD_ALLDC_BATCH 1
 #endif
 #ifndef ODSGD_ALLDC_UNROLL
 #define ODSGD_ALLDC_UNROLL 1
+#endif
+#ifndef ODSGD_ALLDCC_UNROLL
+#define ODSGD_ALLDCC_UNROLL 2
+#endif
+// Block size of the all-workers variants with a delay-compensated or momentum local rule.
+#ifndef ODSGD_ALLDC_BLOCK
+#define ODSGD_ALLDC_BLOCK 128
 #endif
 // 1: one worker's Eq. 4 update in the pass: its previous local weights are fetched with the
 // weights at the top of the tile instead of after the gradient sum (+1.2 % measured).  Not done
@@ -99,6 +112,7 @@ constexpr int kAllSgdBatch = ODSGD_ALLSGD_BATCH;
 constexpr int kAllSgdUnroll = ODSGD_ALLSGD_UNROLL;
 constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
 constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
+constexpr int kAllDcCUnroll = ODSGD_ALLDCC_UNROLL;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
 constexpr bool kOneDcEarly = ODSGD_ONE_DC_EARLY != 0;
 #if ODSGD_MIN_CTAS > 0
@@ -150,7 +164,15 @@ __host__ __device__ constexpr int server_shape_for(int n_workers) {
 // touches three arenas per worker: registers are the scarce resource there).  The kernel and
 // the host-side grid sizing both take the tile from here.
 __host__ __device__ constexpr int server_vectors_per_thread(int local_mode, int rule, int ub) {
-    return local_mode != kLocalAll ? ub : (rule != ODSGD_LOCAL_SGD ? kAllDcUnroll : kAllSgdUnroll);
+    return local_mode != kLocalAll      ? ub
+           : rule == ODSGD_LOCAL_SGD    ? kAllSgdUnroll
+           : rule == ODSGD_LOCAL_DC_C   ? kAllDcCUnroll
+                                        : kAllDcUnroll;
+}
+
+// Threads per CTA the host launches by default.
+__host__ __device__ constexpr int server_default_block(int local_mode, int rule) {
+    return local_mode == kLocalAll && rule != ODSGD_LOCAL_SGD ? ODSGD_ALLDC_BLOCK : kDefaultBlock;
 }
 
 struct LocalParams {

@@ -156,6 +156,12 @@ class PeerExchange:
     def fence(self) -> None:
         self._dist.all_reduce(self._token, group=self.group)
 
+    def quiesce(self) -> None:
+        """Call on every rank before the buffers are dropped: once it returns, no rank has a
+        kernel in flight that reads or writes another rank's memory."""
+        self.fence()
+        torch.cuda.current_stream().synchronize()
+
 
 def shard_views(layout: ShardLayout, rank: int, recv: Sequence[torch.Tensor]) -> List[torch.Tensor]:
     """The N per-worker shard buffers of rank `rank`, as views into its receive buffers, in worker

@@ -340,6 +340,7 @@ def test_single_rank_symmetric_memory_runs_the_direct_exchange(cuda_device):
             assert torch.equal(sh.weights(), ref.weights()) and torch.equal(sh.v[:n], v)
             for j in range(3):
                 assert torch.equal(sh.train_weights(j), ref.train_weights(j))
+        ex.quiesce()
         sh.close()
         ref.close()
     finally:
