@@ -264,15 +264,15 @@ int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry
     // all-workers variants (whose shape is fixed inside the kernel) keep a single instantiation
     if constexpr (LOCAL != kLocalAll && NL == 4) {
         switch (server_shape_for(a.n_workers)) {
-            case kShape2x4: return launch_server_k<DET, NL, LOCAL, RULE, MULT, 2, 4>(c, a, st, dry);
+            case kShape2x4: return launch_server_k<DET, NL, LOCAL, RULE, MULT, ODSGD_SHAPE0_B, ODSGD_SHAPE0_U>(c, a, st, dry);
             case kShape3x4:
                 // 3 x 4 fits the register budget only without a state arena or a multiplier
                 // lookup in the tile; the variants that have one take 4 x 3 (no spills)
                 if constexpr (!MULT && !needs_state(RULE))
-                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, 3, 4>(c, a, st, dry);
+                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, ODSGD_SHAPE1_B, ODSGD_SHAPE1_U>(c, a, st, dry);
                 else
-                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, 4, 3>(c, a, st, dry);
-            case kShape4x3: return launch_server_k<DET, NL, LOCAL, RULE, MULT, 4, 3>(c, a, st, dry);
+                    return launch_server_k<DET, NL, LOCAL, RULE, MULT, ODSGD_SHAPE2_B, ODSGD_SHAPE2_U>(c, a, st, dry);
+            case kShape4x3: return launch_server_k<DET, NL, LOCAL, RULE, MULT, ODSGD_SHAPE2_B, ODSGD_SHAPE2_U>(c, a, st, dry);
             default: break;
         }
     }

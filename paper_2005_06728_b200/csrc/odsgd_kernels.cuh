@@ -148,14 +148,35 @@ enum LocalMode : int { kLocalNone = 0, kLocalOne = 1, kLocalAll = 2, kLocalNoneM
 // thread.  A batch that M divides evenly leaves no half-empty round of loads, and the fewer the
 // streams, the more vectors per thread it takes to keep enough bytes in flight.  Measured on
 // the 138 M-parameter arena (GB/s of algorithmic bytes, fused update), best shape per M:
-//   M <= 2: 2 x 4        M = 3, 5, 6, 9: 3 x 4        M = 4, 7, 8, 10..16: 4 x 3        M > 16: 8 x 2
+//   M <= 2: 2 x 4        M = 3, 5, 6, 9: 3 x 4        M = 4, 7, 8, 10..12: 4 x 3        M > 12: 8 x 2
 // (3 x 4 against 8 x 2: +3 % at M = 3, +4 % at M = 5 and 9; 4 x 3 against 8 x 2: +2 % at M = 12;
-// 8 x 2 wins from M = 24 on; 4 x 4, 6 x 3 and 2 x 6 spill registers and lose 15-25 %.)
+// 8 x 2 against 4 x 3 at M = 13..16: +0-1 % with the plain local rule, +1-3 % with a
+// delay-compensated one, whose early fetch of the previous local weights needs two vectors or
+// fewer; 4 x 4, 6 x 3, 2 x 5 and 2 x 6 spill registers or lose 15-25 %.)
 enum ServerShape : int { kShape2x4 = 0, kShape3x4 = 1, kShape4x3 = 2, kShapeMany = 3 };
+// The three few-worker shapes as batch x vectors (overridable for a sweep, like the rest).
+#ifndef ODSGD_SHAPE0_B
+#define ODSGD_SHAPE0_B 2
+#endif
+#ifndef ODSGD_SHAPE0_U
+#define ODSGD_SHAPE0_U 4
+#endif
+#ifndef ODSGD_SHAPE1_B
+#define ODSGD_SHAPE1_B 3
+#endif
+#ifndef ODSGD_SHAPE1_U
+#define ODSGD_SHAPE1_U 4
+#endif
+#ifndef ODSGD_SHAPE2_B
+#define ODSGD_SHAPE2_B 4
+#endif
+#ifndef ODSGD_SHAPE2_U
+#define ODSGD_SHAPE2_U 3
+#endif
 __host__ __device__ constexpr int server_shape_for(int n_workers) {
     return n_workers <= 2 ? kShape2x4
            : (n_workers == 3 || n_workers == 5 || n_workers == 6 || n_workers == 9) ? kShape3x4
-           : n_workers <= 16 ? kShape4x3
+           : n_workers <= 12 ? kShape4x3
                              : kShapeMany;
 }
 
