@@ -90,3 +90,23 @@ def test_algorithmic_bytes():
     assert ab("local", P, 8) == 3 * 4 * P and ab("asgd", P, 8) == 5 * 4 * P
     assert ab("fused", P, 8) == 13 * 4 * P, "(M + 3) read + 2 written, times 4P"
     assert ab("fused", P, 8, n_locals=8) == 20 * 4 * P
+
+
+def test_profiled_traffic_constants_match_the_committed_capture():
+    """bench.py carries the traffic ratio and the kernel-source hash of the ncu capture as
+    constants; they must be the ones the profile summary records, and the traffic is only
+    reported while the kernel source still is the profiled one."""
+    import hashlib
+    import importlib.util
+    import re
+
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_m32_resnet50_arena.md")).read()
+    assert float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1)) == bench.PROFILED_TRAFFIC_RATIO
+    assert re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1) == bench.PROFILED_KERNEL_SHA256
+    src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
+    current = hashlib.sha256(src).hexdigest() == bench.PROFILED_KERNEL_SHA256
+    got = bench.measured_traffic(1000)
+    assert got == (bench.PROFILED_TRAFFIC_RATIO * 1000 if current else None)
