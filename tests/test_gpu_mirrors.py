@@ -175,3 +175,48 @@ def test_mirror_tables_are_validated(cuda_device):
         c3.set_weight_mirrors([mk()], None)
     assert e.value.code == binding.ERR_STATE
     c3.close()
+
+
+def test_gradients_and_mirrors_outside_device_memory(cuda_device):
+    """The kernel reaches memory that is not this GPU's own with the same plain loads and stores:
+    here page-locked host memory, which the device addresses over the bus under the process's
+    unified addressing - the one kind of non-local memory a single-GPU machine offers.  One
+    gradient is read from there and one mirror per weight half is written there.  Raw pointers,
+    so this goes through the C entry points directly."""
+    n, M = 50_003, 3
+    wl = W.ragged_workload([n], n_workers=M, lr=0.1, local_lr=0.05, momentum=0.9, wd=1e-3, seed=21)
+    w = W.make_weights(wl, DEV)[:n].clone()
+    v, wb = torch.zeros(n, device=DEV), torch.zeros(n, device=DEV)
+    ctx = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd, w_b=wb)
+    lib, h = binding.load_library(), ctx._h
+    host_g = torch.empty(n, dtype=torch.float32).pin_memory()
+    host_ma = torch.full((n,), POISON, dtype=torch.float32).pin_memory()
+    host_mb = torch.full((n,), POISON, dtype=torch.float32).pin_memory()
+    dev_ma, dev_mb = torch.zeros(n, device=DEV), torch.zeros(n, device=DEV)
+    assert all(t.data_ptr() % 16 == 0 for t in (host_g, host_ma, host_mb))
+    ta = binding._ptr_table([dev_ma.data_ptr(), host_ma.data_ptr()])
+    tb = binding._ptr_table([dev_mb.data_ptr(), host_mb.data_ptr()])
+    ctx.check(lib.odsgd_set_weight_mirrors(h, ta, tb, 2))
+    dev_g = [torch.empty(n, device=DEV) for _ in range(M)]
+    table = binding._ptr_table([dev_g[0].data_ptr(), host_g.data_ptr(), dev_g[2].data_ptr()])
+    w_ref, v_ref = w.cpu().numpy().copy(), v.cpu().numpy().copy()
+    stream = torch.cuda.current_stream().cuda_stream
+    for it in range(3):
+        gh = []
+        for m in range(M):
+            g = W.make_grad(wl, m, it, DEV)[:n]
+            if m == 1:
+                host_g.copy_(g)
+            else:
+                dev_g[m].copy_(g)
+            gh.append(g.cpu().numpy())
+        torch.cuda.synchronize()
+        ctx.check(lib.odsgd_global_update(h, table, stream))
+        torch.cuda.synchronize()
+        oracle.global_update(gh, w_ref, v_ref, lr=wl.lr, momentum=wl.momentum, wd=wl.wd)
+        cur = w if it % 2 else wb
+        assert_bits(cur.cpu().numpy(), w_ref, f"weights, iteration {it}")
+        host_m, dev_m = (host_ma, dev_ma) if it % 2 else (host_mb, dev_mb)
+        assert_bits(host_m.numpy(), w_ref, f"mirror in host memory, iteration {it}")
+        assert_bits(dev_m.cpu().numpy(), w_ref, f"mirror in device memory, iteration {it}")
+    ctx.close()
