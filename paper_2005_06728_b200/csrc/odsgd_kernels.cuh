@@ -73,22 +73,27 @@ namespace odsgd {
 #ifndef ODSGD_ALLDC_BLOCK
 #define ODSGD_ALLDC_BLOCK 128
 #endif
-// 1: one worker's Eq. 4 update in the pass: its previous local weights are fetched with the
-// weights at the top of the tile instead of after the gradient sum (+1.2 % measured).  Not done
-// for the rules with a state arena: two more vectors per tile pushed the kernel into spills
-// (Eq. 5-6: -3 %).  Issuing worker m + 1's loads ahead of worker m's stores in the all-workers
-// variants (a software pipeline over the workers) was measured too and lost 1-3 %.
+// One worker's delay-compensated or momentum local update in the pass: where its extra arenas
+// are read and where it is computed.
+//   ODSGD_ONE_INLINE    the update is computed and stored the moment that worker's gradient comes
+//                       by in the sum, its extra arenas fetched with the weights at the top of
+//                       the tile, instead of after the server rule behind one more dependent
+//                       round of loads: 0 never, 1 for the rules with a state arena, 2 for Eq. 4
+//                       as well, 3 for every rule.  Measured against 0 (fused update, one worker):
+//                       Eq. 4 +8 % at M = 8, +16 % at M = 4, +2 % at M = 16; Eq. 5-6 +6 %, +9 %,
+//                       +3.5 % (although 16-48 bytes spill); local momentum +7.5 %, +13 %, +3 %;
+//                       the plain rule within +-0.5 % (it has no extra arena to wait for).
+//   ODSGD_ONE_DC_EARLY  only where the update is not inline: Eq. 4's previous local weights are
+//                       fetched at the top of the tile but used after the server rule: 0 never,
+//                       1 with two vectors per thread or fewer, 2 always (ties with inline, 0.4 %
+//                       ahead at M = 16, but spills up to 192 bytes in the 3 x 4 shape).
+// Issuing worker m + 1's loads ahead of worker m's stores in the all-workers variants (a software
+// pipeline over the workers) was measured too and lost 1-3 %.
 #ifndef ODSGD_ONE_DC_EARLY
 #define ODSGD_ONE_DC_EARLY 1
 #endif
-// One worker's local update in the pass, computed and stored the moment that worker's gradient
-// comes by in the sum (its state fetched at the top of the tile) instead of after the server
-// rule: 0 never, 1 for local momentum SGD, 2 for every rule with an extra arena, 3 for every
-// rule.  Measured (fused update, one worker): local momentum +7.5 % at M = 8 (61 M parameters),
-// +13-15 % at M = 1..4, +3 % at M = 16, +1 % at M = 32; Eq. 4 and Eq. 5-6 -1 to -6 %; the plain
-// rule within +-0.5 %.
 #ifndef ODSGD_ONE_INLINE
-#define ODSGD_ONE_INLINE 1
+#define ODSGD_ONE_INLINE 2
 #endif
 // Local and ASGD kernels: vectors per thread per tile.
 #ifndef ODSGD_SMALL_UNROLL
@@ -123,7 +128,7 @@ constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
 constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
 constexpr int kAllDcCUnroll = ODSGD_ALLDCC_UNROLL;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
-constexpr bool kOneDcEarly = ODSGD_ONE_DC_EARLY != 0;
+constexpr int kOneDcEarly = ODSGD_ONE_DC_EARLY;
 constexpr int kOneInline = ODSGD_ONE_INLINE;
 #if ODSGD_MIN_CTAS > 0
 #define ODSGD_SERVER_BOUNDS __launch_bounds__(ODSGD_MAX_BLOCK, ODSGD_MIN_CTAS)
@@ -437,21 +442,29 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                                                const bool (&ok)[U], TensorCursor& cur) {
     using O = Op<DET>;
     Vec<NL> w[U], v[U], s[U], gl[U];
-    // one worker's Eq. 4 rule: its previous local weights are fetched early (only with two vectors
-    // per thread or fewer: the wide few-worker shape has no registers to spare)
+    // one worker's local update with extra arenas: inline in the sum, or fetched early (see
+    // ODSGD_ONE_INLINE / ODSGD_ONE_DC_EARLY)
     constexpr bool kInline = LOCAL == kLocalOne &&
                              (kOneInline == 3 || (kOneInline == 2 && RULE != ODSGD_LOCAL_SGD) ||
-                              (kOneInline == 1 && RULE == ODSGD_LOCAL_MOMENTUM));
+                              (kOneInline == 1 && needs_state(RULE)));
     constexpr bool kOneDc = LOCAL == kLocalOne && (needs_prev(RULE) || needs_state(RULE)) &&
-                            (kInline || (!needs_state(RULE) && kOneDcEarly && U <= 2));
+                            (kInline || (!needs_state(RULE) && kOneDcEarly == 1 && U <= 2) ||
+                             (!needs_state(RULE) && kOneDcEarly == 2));
     Vec<NL> xe[kOneDc ? U : 1], mse[kOneDc ? U : 1];
+    // Where a worker's previous local weights are read from.  On the first delayed step the
+    // gradient was taken on w_bak itself, so x_prev := w_bak: the same loads, pointed at the
+    // weights.  (A pointer select, not a conditional load: with the choice made per load, the
+    // loads of a tile were no longer issued together, which cost the one-worker Eq. 4 / Eq. 5-6
+    // passes 3-16 % and the local kernel 16-42 %.)  Every element's x_prev is read before the
+    // same thread stores that element of w_out, so the in-place layout reads the old weights.
+    const float* xprev_one = a.lp.first ? a.w_in : a.x[0];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
         if (ok[u]) {
             w[u] = load_stream<NL>(a.w_in + off[u]);
             v[u] = load_stream<NL>(a.v + off[u]);
             if (kOneDc) {
-                if (needs_prev(RULE)) xe[u] = a.lp.first ? w[u] : load_stream<NL>(a.x[0] + off[u]);
+                if (needs_prev(RULE)) xe[u] = load_stream<NL>(xprev_one + off[u]);
                 if (needs_state(RULE)) mse[u] = load_stream<NL>(a.ms[0] + off[u]);
             }
         }
@@ -479,7 +492,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
 #pragma unroll
                         for (int u = 0; u < U; ++u) {
                             if (ok[u]) {
-                                if (needs_prev(RULE)) xv[j][u] = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+                                if (needs_prev(RULE)) xv[j][u] = load_stream<NL>((a.lp.first ? a.w_in : xp) + off[u]);
                                 if (needs_state(RULE)) msv[j][u] = load_stream<NL>(a.ms[m0 + j] + off[u]);
                             }
                         }
@@ -557,7 +570,7 @@ __device__ __forceinline__ void server_vectors(const ServerArgs& a, const unsign
                 xv = xe[u];
                 msv = mse[u];
             } else {
-                if (needs_prev(RULE)) xv = a.lp.first ? w[u] : load_stream<NL>(xp + off[u]);
+                if (needs_prev(RULE)) xv = load_stream<NL>(xprev_one + off[u]);
                 if (needs_state(RULE)) msv = load_stream<NL>(a.ms[0] + off[u]);
             }
 #pragma unroll
@@ -625,7 +638,7 @@ __device__ __forceinline__ void local_vectors(const LocalArgs& a, const unsigned
         if (ok[u]) {
             w[u] = SERVER ? load_stream<NL>(a.w_bak + off[u]) : load_grad<NL>(a.w_bak + off[u]);
             g[u] = load_grad<NL>(a.g + off[u]);
-            if (needs_prev(RULE)) xv[u] = a.lp.first ? w[u] : load_stream<NL>(a.x + off[u]);
+            if (needs_prev(RULE)) xv[u] = load_stream<NL>((a.lp.first ? a.w_bak : a.x) + off[u]);
             if (needs_state(RULE)) msv[u] = load_stream<NL>(a.ms + off[u]);
         }
     }
