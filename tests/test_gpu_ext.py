@@ -125,9 +125,12 @@ def _dc_oracle_local(rule, wp, g, x_prev, ms, llr, lam, m, eps):
 @pytest.mark.parametrize("rule", [binding.LOCAL_SGD, binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
                          ids=["sgd", "dc_c", "dc_a", "momentum"])
 @pytest.mark.parametrize("wp", [0, 1, 3])
-def test_algorithm2_state_machine(cuda_device, rule, wp):
+@pytest.mark.parametrize("layout", ["pingpong", "inplace"])
+def test_algorithm2_state_machine(cuda_device, rule, wp, layout):
     """odsgd_step: wp SSGD iterations, then fused global + local updates; the first local
-    update (iteration wp) sees no delay; the chain x_prev -> x runs through the local arenas."""
+    update (iteration wp) sees no delay; the chain x_prev -> x runs through the local arenas.
+    In the in-place layout the weights are overwritten by the same pass that, at iteration wp,
+    reads them a second time as x_prev."""
     wl = W.ragged_workload([3000, 17, 40_004, 5], n_workers=3, lr=0.05, local_lr=0.04, momentum=0.9, wd=1e-3)
     M, n = 3, wl.arena_len
     lam, m_, eps = 0.5, 0.95, 1e-7
@@ -137,7 +140,8 @@ def test_algorithm2_state_machine(cuda_device, rule, wp):
     local = [torch.full_like(w, 777.0) for _ in range(M)]  # junk: must never be read as x_prev at iteration wp
     msq = [torch.zeros_like(w) for _ in range(M)]
     ctx = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
-                        w_b=w_b, local=local, tensor_offsets=wl.offsets, flags=binding.FLAG_DETERMINISTIC)
+                        w_b=w_b if layout == "pingpong" else None, w_delayed=None if layout == "pingpong" else w_b,
+                        local=local, tensor_offsets=wl.offsets, flags=binding.FLAG_DETERMINISTIC)
     has_state = rule in (binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM)
     ctx.set_local_rule(rule, lam, m_, eps, msq if has_state else None)
     ctx.set_warmup(wp)
