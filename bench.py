@@ -54,7 +54,7 @@ def hbm_peak():
 # dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of that launch, and the
 # SHA-256 of csrc/odsgd_kernels.cuh (kernels and launch shapes) at the time of the capture.
 PROFILED_TRAFFIC_RATIO = 0.998
-PROFILED_KERNEL_SHA256 = "feb053ba262cfc1ed5dd974b1a9f5d9cfb6a95146634c506f817186dcbd5ebe2"
+PROFILED_KERNEL_SHA256 = "f703dab00eb758d801c72623e417943dbe5a790e907b4d15dc9afb47cbaf79d6"
 
 
 def measured_traffic(step_bytes):

@@ -53,7 +53,7 @@ namespace odsgd {
 // 138 M-parameter arena, equal on the others; 3 x 4 and 2 x 5 tie, 1 x 4, 1 x 6, 2 x 6 lose 3-8 %);
 // Eq. 4: one worker per round, 2 vectors, 128-thread CTAs (+2 % over 1 vector x 256 threads; 3
 // vectors lose 4 %); Eq. 5-6 and local momentum: one worker, one vector, 128-thread CTAs (+2 %
-// for Eq. 5-6; two workers per round lose 15-20 %, two vectors 3-10 %).
+// for Eq. 5-6; two or four workers per round change it by less than 1 %, two vectors cost 3-4 %).
 #ifndef ODSGD_ALLSGD_BATCH
 #define ODSGD_ALLSGD_BATCH 2
 #endif
