@@ -92,11 +92,10 @@ def test_algorithmic_bytes():
     assert ab("fused", P, 8, n_locals=8) == 20 * 4 * P
 
 
-def test_profiled_traffic_constants_match_the_committed_capture():
-    """bench.py carries the traffic ratio and the kernel-source hash of the ncu capture as
+def test_profiled_traffic_constants_match_the_committed_capture(tmp_path):
+    """bench.py carries the traffic ratio and the kernel-source digest of the ncu capture as
     constants; they must be the ones the profile summary records, and the traffic is only
-    reported while the kernel source still is the profiled one."""
-    import hashlib
+    reported while the kernel source still is the profiled one (comments aside)."""
     import importlib.util
     import re
 
@@ -105,8 +104,14 @@ def test_profiled_traffic_constants_match_the_committed_capture():
     spec.loader.exec_module(bench)
     note = open(os.path.join(ROOT, "profiles", "server_kernel_fused_m32_resnet50_arena.md")).read()
     assert float(re.search(r"^traffic_ratio:\s*([0-9.]+)", note, re.M).group(1)) == bench.PROFILED_TRAFFIC_RATIO
-    assert re.search(r"^kernel_source_sha256:\s*([0-9a-f]+)", note, re.M).group(1) == bench.PROFILED_KERNEL_SHA256
-    src = open(os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh"), "rb").read()
-    current = hashlib.sha256(src).hexdigest() == bench.PROFILED_KERNEL_SHA256
+    assert re.search(r"^kernel_source_digest:\s*([0-9a-f]+)", note, re.M).group(1) == bench.PROFILED_KERNEL_DIGEST
+    current = bench.kernel_source_digest() == bench.PROFILED_KERNEL_DIGEST
     got = bench.measured_traffic(1000)
     assert got == (bench.PROFILED_TRAFFIC_RATIO * 1000 if current else None)
+    # the digest ignores comments and blank lines, and nothing else
+    src = open(bench.KERNEL_SOURCE, encoding="utf-8").read()
+    a = tmp_path / "a.cuh"
+    a.write_text("// a new remark\n\n" + src.replace("#pragma once", "#pragma once  // reworded"))
+    assert bench.kernel_source_digest(str(a)) == bench.kernel_source_digest()
+    a.write_text(src.replace("#define ODSGD_BATCH 8", "#define ODSGD_BATCH 4"))
+    assert bench.kernel_source_digest(str(a)) != bench.kernel_source_digest()
