@@ -182,6 +182,60 @@ def test_algorithm2_state_machine(cuda_device, rule, wp, layout):
 
 @pytest.mark.parametrize("rule", [binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
                          ids=["dc_c", "dc_a", "momentum"])
+@pytest.mark.parametrize("M", [1, 2, 3, 5, 8, 12, 13, 16, 33])
+@pytest.mark.parametrize("layout", ["pingpong", "inplace"])
+def test_fused_one_worker_with_extra_arenas_over_worker_counts(cuda_device, rule, M, layout):
+    """One worker's Eq. 4 / Eq. 5-6 / momentum update inside the server pass, for every launch
+    shape of the kernel (the worker counts), for the first, a middle and the last worker (the
+    update is computed where that worker's gradient comes by in the sum), on a ragged arena of
+    several tiles, with per-tensor multipliers on the server rule in one of the steps.  The
+    chain x_prev -> x and the state arenas run through three calls; bit for bit against the
+    oracle."""
+    wl = W.ragged_workload([9_001, 7, 11_000, 3], n_workers=M, lr=0.05, local_lr=0.04, momentum=0.9, wd=1e-3, seed=M)
+    n = wl.arena_len
+    lam, m_, eps = 0.5, 0.95, 1e-7
+    has_state = rule in (binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM)
+    workers = sorted({0, M // 2, M - 1})
+    w = W.make_weights(wl, DEV)
+    v = W.make_momentum(wl, DEV)
+    other = torch.zeros_like(w)
+    local = [w.clone() + 0.01 * (i + 1) if i in workers else None for i in range(M)]
+    msq = [torch.zeros_like(w) if i in workers else None for i in range(M)]
+    ctx = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                        w_b=other if layout == "pingpong" else None, w_delayed=None if layout == "pingpong" else other,
+                        local=local, tensor_offsets=wl.offsets)
+    ctx.set_local_rule(rule, lam, m_, eps, msq if has_state else None)
+    w_ref, v_ref = w.cpu().numpy().copy(), v.cpu().numpy().copy()
+    x_ref = {i: local[i].cpu().numpy().copy() for i in workers}
+    ms_ref = {i: np.zeros(n, np.float32) for i in workers}
+    lr_mult = np.asarray([1.0, 0.0, 2.0, 0.5], np.float32)
+    wd_mult = np.asarray([1.0, 0.0, 1.0, 0.0], np.float32)
+    hp = dict(lr=wl.lr, momentum=wl.momentum, wd=wl.wd)
+    for it, wk in enumerate(workers + [workers[0]]):
+        grads = W.make_grads(wl, it, DEV)
+        gh = [g.cpu().numpy() for g in grads]
+        mult = it == 1
+        ctx.set_tensor_multipliers(lr_mult.tolist() if mult else None, wd_mult.tolist() if mult else None)
+        ctx.fused_update(grads, wk)
+        wprev = np.empty_like(w_ref)
+        if mult:
+            oracle.global_update_mult(gh, w_ref, v_ref, offsets=wl.offsets, lr_mult=lr_mult, wd_mult=wd_mult,
+                                      w_prev=wprev, **hp)
+        else:
+            oracle.global_update(gh, w_ref, v_ref, w_prev=wprev, **hp)
+        x_ref[wk] = _dc_oracle_local(rule, wprev, gh[wk], x_ref[wk], ms_ref[wk], wl.local_lr, lam, m_, eps)
+        torch.cuda.synchronize()
+        assert_bits(ctx.weights().cpu().numpy(), w_ref, f"w, call {it}")
+        assert_bits(v.cpu().numpy(), v_ref, f"v, call {it}")
+        for i in workers:  # the updated worker's arenas moved on, the others' are untouched
+            assert_bits(local[i].cpu().numpy(), x_ref[i], f"x[{i}], call {it} (updated worker {wk})")
+            if has_state:
+                assert_bits(msq[i].cpu().numpy(), ms_ref[i], f"state[{i}], call {it}")
+    ctx.close()
+
+
+@pytest.mark.parametrize("rule", [binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
+                         ids=["dc_c", "dc_a", "momentum"])
 def test_separate_dc_local_update_equals_fused(cuda_device, rule):
     wl = W.ragged_workload([10_000, 33], n_workers=2)
     ctxs = []
