@@ -262,7 +262,13 @@ template <bool DET, int NL, int LOCAL, int RULE, bool MULT>
 int launch_server_m(odsgd_ctx* c, const ServerArgs& a, cudaStream_t st, bool dry) {
     // the shape follows the worker count on the 128-bit path; the scalar fallback and the
     // all-workers variants (whose shape is fixed inside the kernel) keep a single instantiation
-    if constexpr (LOCAL != kLocalAll && NL == 4) {
+    if constexpr (LOCAL == kLocalOne && NL == 4 && needs_prev(RULE) && needs_state(RULE)) {
+        // one worker's Eq. 5-6 update carries two more vectors per tile vector than the other
+        // rules (previous local weights and mean square): the wide few-worker shapes spill and
+        // the narrower ones win (2 x 3 against 2 x 4: +15-18 % at M <= 2, +3 % at M = 4; 8 x 2
+        // against 3 x 4 / 4 x 3: +6 % at M = 6, +4 % at M = 8, +1 % at M = 12)
+        if (a.n_workers <= 4) return launch_server_k<DET, NL, LOCAL, RULE, MULT, 2, 3>(c, a, st, dry);
+    } else if constexpr (LOCAL != kLocalAll && NL == 4) {
         switch (server_shape_for(a.n_workers)) {
             case kShape2x4: return launch_server_k<DET, NL, LOCAL, RULE, MULT, ODSGD_SHAPE0_B, ODSGD_SHAPE0_U>(c, a, st, dry);
             case kShape3x4:
