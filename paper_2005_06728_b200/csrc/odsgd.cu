@@ -326,7 +326,7 @@ int launch_server(odsgd_ctx* c, const ServerArgs& a, int lanes, int local_mode, 
 
 template <bool DET, int NL, int RULE, bool SERVER>
 int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
-    const int block = c->block_threads > 0 ? c->block_threads : kDefaultLocalBlock;
+    const int block = c->block_threads > 0 ? c->block_threads : local_default_block(RULE);
     auto kernel = local_kernel<DET, NL, RULE, SERVER>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
     launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kLocalCtasPerSm), block, st, a);
