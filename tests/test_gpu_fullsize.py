@@ -16,6 +16,11 @@ M gradients is copied to the host, the oracle advances its own copy of the state
 and the library's result for the chunk is compared bit by bit.  The host never holds more than
 one chunk of the gradients; the three independent oracle trajectories of a chunk run in three
 threads (the oracle itself stays single-threaded code).
+
+The local rules with extra arenas (Eq. 4, Eq. 5-6, local momentum: the flavours the paper trained
+its CIFAR-10 and ImageNet models with) get the same treatment on the AlexNet- and ResNet-50-shaped
+sets: three iterations, every element, the update of one worker inside the server pass and the
+update of three workers in the all-workers pass, each chained through its own arenas.
 """
 from concurrent.futures import ThreadPoolExecutor
 
@@ -165,3 +170,91 @@ def test_resnet56_ssgd_and_asgd_full_run(cuda_device):
 def test_lenet5_every_rule_full_run(cuda_device):
     wl = W.workload("lenet5")
     _run_config("lenet5", wl.iterations, wl.iterations)
+
+
+RULES = {"dc_c": binding.LOCAL_DC_C, "dc_a": binding.LOCAL_DC_A, "momentum": binding.LOCAL_MOMENTUM}
+LAM, DECAY, EPS = 0.04, 0.95, 1e-7
+
+
+def _oracle_local(rule, bak, g, x_prev, state, llr):
+    """One worker's local update on a chunk; `state` (mean square or velocity) is updated in place."""
+    if rule == "dc_c":
+        return oracle.local_update_dc_c(bak, g, x_prev, local_lr=llr, lam=LAM)
+    if rule == "dc_a":
+        return oracle.local_update_dc_a(bak, g, x_prev, state, local_lr=llr, lam=LAM, m=DECAY, eps=EPS)
+    return oracle.local_update_momentum(bak, g, state, local_lr=llr, momentum=DECAY, wd=LAM)
+
+
+def _run_local_rules(name, iterations):
+    wl = W.workload(name)
+    n, M = wl.arena_len, wl.n_workers
+    free, _ = torch.cuda.mem_get_info()
+    if free < (M + 48) * n * 4 * 1.1:
+        pytest.skip("not enough device memory")
+    last, some = M - 1, (0, M // 2, M - 1)
+    w0 = W.make_weights(wl, DEV)
+    ctxs = {}
+    for rule, rid in RULES.items():
+        for kind, who in (("one", (last,)), ("some", some)):
+            w, v, other = w0.clone(), torch.zeros_like(w0), torch.zeros_like(w0)
+            local = [w0.clone() if m in who else None for m in range(M)]
+            state = [torch.zeros_like(w0) if m in who else None for m in range(M)]
+            c = binding.Odsgd(w, v, n_workers=M, lr=wl.lr, local_lr=wl.local_lr, momentum=wl.momentum, wd=wl.wd,
+                              w_b=other, local=local, tensor_offsets=wl.offsets)
+            c.set_local_rule(rid, LAM, DECAY, EPS, state if rule != "dc_c" else None)
+            ctxs[rule, kind] = (c, v, local, state)
+    # the oracle's copies: one server trajectory (it is the same in all six contexts), and per
+    # rule and context the local weights and states of the workers that context updates
+    od_w, od_v = w0.cpu().numpy().copy(), np.zeros(n, np.float32)
+    hx = {(r, k, m): od_w.copy() for r in RULES for k, who in (("one", (last,)), ("some", some)) for m in who}
+    hs = {key: np.zeros(n, np.float32) for key in hx}
+    hp = dict(lr=wl.lr, momentum=wl.momentum, wd=wl.wd)
+    grads = [torch.empty(n, dtype=torch.float32, device=DEV) for _ in range(M)]
+    sg, pads = W.sigma_arena(wl, DEV), W.pad_mask(wl, DEV)
+    stage = torch.empty((M, min(CHUNK, n)), dtype=torch.float32).pin_memory()
+    pool = ThreadPoolExecutor(3)
+    for it in range(iterations):
+        for m in range(M):
+            W.make_grad(wl, m, it, DEV, out=grads[m], _sigma=sg, _pads=pads)
+        for (rule, kind), (c, _, _, _) in ctxs.items():
+            c.fused_update(grads, last if kind == "one" else -1)
+        torch.cuda.synchronize()
+        for a in range(0, n, CHUNK):
+            b = min(a + CHUNK, n)
+            for m in range(M):
+                stage[m, :b - a].copy_(grads[m][a:b], non_blocking=True)
+            torch.cuda.synchronize()
+            gh = [stage[m, :b - a].numpy() for m in range(M)]
+            bak = np.empty(b - a, np.float32)
+            oracle.global_update(gh, od_w[a:b], od_v[a:b], w_prev=bak, **hp)
+
+            def rule_job(rule):
+                for (r, k, m) in hx:
+                    if r == rule:
+                        hx[r, k, m][a:b] = _oracle_local(rule, bak, gh[m], hx[r, k, m][a:b].copy(), hs[r, k, m][a:b],
+                                                         wl.local_lr)
+
+            for j in [pool.submit(rule_job, r) for r in RULES]:
+                j.result()
+            for (rule, kind), (c, v, local, state) in ctxs.items():
+                tag = f"{name} {rule}/{kind} it {it} [{a}:{b}]"
+                assert_bits(c.weights()[a:b].cpu().numpy(), od_w[a:b], f"w {tag}")
+                assert_bits(v[a:b].cpu().numpy(), od_v[a:b], f"v {tag}")
+                for m in ((last,) if kind == "one" else some):
+                    assert_bits(local[m][a:b].cpu().numpy(), hx[rule, kind, m][a:b], f"x[{m}] {tag}")
+                    if rule != "dc_c":
+                        assert_bits(state[m][a:b].cpu().numpy(), hs[rule, kind, m][a:b], f"state[{m}] {tag}")
+    pool.shutdown()
+    for c, _, _, _ in ctxs.values():
+        assert c.launch_count == iterations
+        c.close()
+    del grads, stage, ctxs
+    torch.cuda.empty_cache()
+
+
+def test_alexnet_local_rules_with_extra_arenas_every_element(cuda_device):
+    _run_local_rules("alexnet", 3)
+
+
+def test_resnet50_local_rules_with_extra_arenas_every_element(cuda_device):
+    _run_local_rules("resnet50", 3)
