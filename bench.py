@@ -54,7 +54,7 @@ def hbm_peak():
 # dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of that launch, and the
 # digest of csrc/odsgd_kernels.cuh (kernels and launch shapes) at the time of the capture.
 PROFILED_TRAFFIC_RATIO = 0.998
-PROFILED_KERNEL_DIGEST = "19887ec870cd4e4ece283a47c495f552faa6c2a5ba885e082ee3aa5dd42223c7"
+PROFILED_KERNEL_DIGEST = "79ef5221ea86938766b44ad7025d7e7348844e0c8d0347dabd87d8e52572d1c4"
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh")
 
 

@@ -329,7 +329,7 @@ int launch_local_t(odsgd_ctx* c, const LocalArgs& a, cudaStream_t st) {
     const int block = c->block_threads > 0 ? c->block_threads : local_default_block(RULE);
     auto kernel = local_kernel<DET, NL, RULE, SERVER>;
     if (resident_cached(c, kernel, block) == 0) return too_wide(c, block);
-    launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kSmallUnroll, kLocalCtasPerSm), block, st, a);
+    launch_kernel<LocalArgs>(kernel, grid_for(c, a.n, NL, block, kLocalUnroll, kLocalCtasPerSm), block, st, a);
     return after_launch(c, "local kernel launch");
 }
 

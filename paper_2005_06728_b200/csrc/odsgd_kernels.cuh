@@ -95,9 +95,14 @@ namespace odsgd {
 #ifndef ODSGD_ONE_INLINE
 #define ODSGD_ONE_INLINE 2
 #endif
-// Local and ASGD kernels: vectors per thread per tile.
+// ASGD kernel / local kernel: vectors per thread per tile.  The local kernel with the plain rule
+// (two streams in, one out) does 1 % better with three than with four on all three large arenas,
+// the ASGD kernel 0.2-0.6 % better with four; two or six lose 0.5-1 % in both.
 #ifndef ODSGD_SMALL_UNROLL
 #define ODSGD_SMALL_UNROLL 4
+#endif
+#ifndef ODSGD_LOCAL_UNROLL
+#define ODSGD_LOCAL_UNROLL 3
 #endif
 // Gradient loads: 0 streaming (ld.global.cs), 1 read-only path (ld.global.nc), 2 default caching,
 // 3 read-only path without L1 allocation and a 256-byte L2 prefetch hint, 4 read-only path without
@@ -128,6 +133,7 @@ constexpr int kAllDcBatch = ODSGD_ALLDC_BATCH;
 constexpr int kAllDcUnroll = ODSGD_ALLDC_UNROLL;
 constexpr int kAllDcCUnroll = ODSGD_ALLDCC_UNROLL;
 constexpr int kSmallUnroll = ODSGD_SMALL_UNROLL;
+constexpr int kLocalUnroll = ODSGD_LOCAL_UNROLL;
 constexpr int kOneDcEarly = ODSGD_ONE_DC_EARLY;
 constexpr int kOneInline = ODSGD_ONE_INLINE;
 #if ODSGD_MIN_CTAS > 0
@@ -628,7 +634,7 @@ __global__ void ODSGD_SERVER_BOUNDS server_kernel(const __grid_constant__ Server
 }
 
 // ------------------------------------------------------------------ local kernel
-// Few streams per element (2-4 reads, 1-2 writes): each thread takes kSmallUnroll vectors per
+// Few streams per element (2-4 reads, 1-2 writes): each thread takes kLocalUnroll vectors per
 // tile and issues all their loads before the first store, which is what a plain copy needs
 // to approach the copy ceiling of the part.
 // SERVER = true is DC-ASGD at the parameter server (Eq. 4 / Eq. 5 applied to an arriving
@@ -663,18 +669,18 @@ template <bool DET, int NL, int RULE, bool SERVER>
 __global__ void local_kernel(const __grid_constant__ LocalArgs a) {
     dependent_launch_prologue();
     const unsigned long long nvec = a.n / NL;
-    const unsigned long long tile = (unsigned long long)blockDim.x * kSmallUnroll;
+    const unsigned long long tile = (unsigned long long)blockDim.x * kLocalUnroll;
     const unsigned long long stride = (unsigned long long)gridDim.x * tile;
     for (unsigned long long base = (unsigned long long)blockIdx.x * tile; base < nvec; base += stride) {
-        unsigned long long off[kSmallUnroll];
-        bool ok[kSmallUnroll];
+        unsigned long long off[kLocalUnroll];
+        bool ok[kLocalUnroll];
 #pragma unroll
-        for (int u = 0; u < kSmallUnroll; ++u) {
+        for (int u = 0; u < kLocalUnroll; ++u) {
             const unsigned long long i = base + (unsigned long long)u * blockDim.x + threadIdx.x;
             ok[u] = i < nvec;
             off[u] = i * NL;
         }
-        local_vectors<DET, NL, RULE, SERVER, kSmallUnroll>(a, off, ok);
+        local_vectors<DET, NL, RULE, SERVER, kLocalUnroll>(a, off, ok);
     }
     if (NL > 1) {
         const unsigned long long done = nvec * NL;
