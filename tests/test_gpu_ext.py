@@ -182,7 +182,7 @@ def test_algorithm2_state_machine(cuda_device, rule, wp, layout):
 
 @pytest.mark.parametrize("rule", [binding.LOCAL_DC_C, binding.LOCAL_DC_A, binding.LOCAL_MOMENTUM],
                          ids=["dc_c", "dc_a", "momentum"])
-@pytest.mark.parametrize("M", [1, 2, 3, 5, 8, 12, 13, 16, 33])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8, 12, 13, 16, 33, 64])
 @pytest.mark.parametrize("layout", ["pingpong", "inplace"])
 def test_fused_one_worker_with_extra_arenas_over_worker_counts(cuda_device, rule, M, layout):
     """One worker's Eq. 4 / Eq. 5-6 / momentum update inside the server pass, for every launch
