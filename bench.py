@@ -54,7 +54,7 @@ def hbm_peak():
 # dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of that launch, and the
 # digest of csrc/odsgd_kernels.cuh (kernels and launch shapes) at the time of the capture.
 PROFILED_TRAFFIC_RATIO = 0.998
-PROFILED_KERNEL_DIGEST = "79ef5221ea86938766b44ad7025d7e7348844e0c8d0347dabd87d8e52572d1c4"
+PROFILED_KERNEL_DIGEST = "29d418ddb2084b4c21b8f33a6d9a255c4ca09cf5975ade67586460aa972cdd87"
 KERNEL_SOURCE = os.path.join(ROOT, "paper_2005_06728_b200", "csrc", "odsgd_kernels.cuh")
 
 

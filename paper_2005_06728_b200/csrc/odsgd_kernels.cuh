@@ -151,12 +151,13 @@ constexpr int kDefaultAsgdBlock = 256;   // ASGD kernel (256 against 512 threads
 // loop depends on how heavy a tile is.  With many gradient streams a tile is hundreds of KB and
 // finer-grained scheduling evens out the tail: 256 per SM (in effect one tile per CTA) measured
 // 0.6-1.9 % faster than 64 from M = 4 up, and than an exactly persistent grid.  The copy-like
-// one-worker pass has light tiles and pays for CTA turnover instead: 16 per SM is 6 % faster
-// than 64 on the 25-61 M-parameter arenas (equal on the 138 M one); two workers sit in between.
+// one-worker pass has light tiles and sits in between: 32 per SM (against 16: +1 % on the 61 M-
+// and 138 M-parameter arenas, equal on the 25 M one; 64 gains another 1 % on the large two and
+// loses 2.4 % on the small one); two workers take 64.
 constexpr int kLocalCtasPerSm = 128;
 constexpr int kAsgdCtasPerSm = 256;
 __host__ __device__ constexpr int server_grid_cap(int n_workers) {
-    return n_workers <= 1 ? 16 : (n_workers == 2 ? 64 : 256);
+    return n_workers <= 1 ? 32 : (n_workers == 2 ? 64 : 256);
 }
 
 // What else the server pass carries: nothing, one worker's local update, every worker's, or -
